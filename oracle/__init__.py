@@ -1,0 +1,121 @@
+"""ctypes front end of the CPU oracle (test infrastructure only).
+
+Nothing under the product package imports this module. Tests, the smoke check
+and the benchmark's CPU-baseline leg do. `build()` compiles `ep_oracle.c` with
+the host C compiler; no CUDA is involved.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from dataclasses import dataclass
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "ep_oracle.c")
+_LIB = os.path.join(_HERE, "libep_oracle.so")
+_lib = None
+
+STATUS_BAD_INDEX = 1
+
+
+def build(force: bool = False) -> str:
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        cmd = ["gcc", "-O2", "-std=c11", "-ffp-contract=off", "-fPIC", "-shared", "-Wall", "-Wextra",
+               "-o", _LIB, _SRC, "-lm"]
+        subprocess.run(cmd, check=True)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        build()
+        _lib = ctypes.CDLL(_LIB)
+    return _lib
+
+
+def _p(a: np.ndarray):
+    return a.ctypes.data_as(ctypes.c_void_p)
+
+
+@dataclass
+class Layout:
+    expert_counts: np.ndarray
+    expert_offsets: np.ndarray
+    rank_rows: np.ndarray
+    rank_row_offsets: np.ndarray
+    src_row_offsets: np.ndarray     # [R, R+1]
+    recv_slot: np.ndarray           # [T, K]
+    pair_slot: np.ndarray           # [T, K]
+    recv_token: np.ndarray          # [N_recv]
+    pair_row: np.ndarray            # [P]
+    pair_token: np.ndarray          # [P]
+    status: int
+
+    @property
+    def n_recv(self) -> int:
+        return int(self.rank_row_offsets[-1])
+
+    @property
+    def n_pairs(self) -> int:
+        return int(self.expert_offsets[-1])
+
+
+def layout(topk_idx: np.ndarray, E: int, R: int) -> Layout:
+    idx = np.ascontiguousarray(topk_idx, dtype=np.int32)
+    T, K = idx.shape
+    i32 = np.int32
+    ec = np.zeros(E, i32); eo = np.zeros(E + 1, i32)
+    rr = np.zeros(R, i32); ro = np.zeros(R + 1, i32)
+    so = np.zeros((R, R + 1), i32)
+    rs = np.full((T, K), -1, i32); ps = np.full((T, K), -1, i32)
+    rt = np.full(max(1, T * min(K, R)), -1, i32)
+    pr = np.full(max(1, T * K), -1, i32); pt = np.full(max(1, T * K), -1, i32)
+    st = np.zeros(1, i32)
+    rc = _load().ep_oracle_layout(T, K, E, R, _p(idx), _p(ec), _p(eo), _p(rr), _p(ro), _p(so),
+                                  _p(rs), _p(ps), _p(rt), _p(pr), _p(pt), _p(st))
+    if rc != 0:
+        raise ValueError("oracle layout: shape outside the definitions (need E % R == 0, T % R == 0)")
+    return Layout(ec, eo, rr, ro, so, rs, ps, rt[: int(ro[-1])], pr[: int(eo[-1])],
+                  pt[: int(eo[-1])], int(st[0]))
+
+
+def dispatch(x_bits: np.ndarray, recv_slot: np.ndarray, recv_rows: int, fill: int = 0) -> np.ndarray:
+    x = np.ascontiguousarray(x_bits, dtype=np.uint16)
+    slot = np.ascontiguousarray(recv_slot, dtype=np.int32)
+    T, H = x.shape
+    K = slot.shape[1]
+    recv = np.full((recv_rows, H), fill, dtype=np.uint16)
+    rc = _load().ep_oracle_dispatch(T, K, H, _p(x), _p(slot), _p(recv), ctypes.c_int64(recv_rows))
+    if rc != 0:
+        raise ValueError("oracle dispatch: slot beyond recv_rows")
+    return recv
+
+
+def combine_f32(out_bits: np.ndarray, slot: np.ndarray, w: np.ndarray) -> np.ndarray:
+    out = np.ascontiguousarray(out_bits, dtype=np.uint16)
+    s = np.ascontiguousarray(slot, dtype=np.int32)
+    wt = np.ascontiguousarray(w, dtype=np.float32)
+    T, K = s.shape
+    H = out.shape[1]
+    y = np.zeros((T, H), dtype=np.uint16)
+    rc = _load().ep_oracle_combine_f32(T, K, H, _p(out), ctypes.c_int64(out.shape[0]), _p(s), _p(wt), _p(y))
+    if rc != 0:
+        raise ValueError("oracle combine: slot beyond out rows")
+    return y
+
+
+def combine_f64(out_bits: np.ndarray, slot: np.ndarray, w: np.ndarray) -> np.ndarray:
+    out = np.ascontiguousarray(out_bits, dtype=np.uint16)
+    s = np.ascontiguousarray(slot, dtype=np.int32)
+    wt = np.ascontiguousarray(w, dtype=np.float32)
+    T, K = s.shape
+    H = out.shape[1]
+    y = np.zeros((T, H), dtype=np.float64)
+    rc = _load().ep_oracle_combine_f64(T, K, H, _p(out), ctypes.c_int64(out.shape[0]), _p(s), _p(wt), _p(y))
+    if rc != 0:
+        raise ValueError("oracle combine: slot beyond out rows")
+    return y
