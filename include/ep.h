@@ -1,0 +1,201 @@
+/*
+ * ep.h -- C ABI of the B200 (sm_100a) routing-aware expert-parallel token
+ * dispatch / combine library.
+ *
+ * The problem, as the paper states it (Section 2.1, "Distributed MoE and expert
+ * parallelism"): a router picks K of E experts for each of T tokens; the experts
+ * are partitioned over R devices ("ranks") and every rank owns a block of the
+ * tokens. Before the expert computation a token's activation must reach every
+ * rank that hosts one of its picked experts (dispatch); afterwards the expert
+ * outputs return to the token's owner and are summed there (combine). This
+ * library implements the routing-aware form (Section 2.1, "Communication
+ * patterns of dispatch and combine"; Section 4.5, "Routing-aware
+ * communication"): only the rows a destination needs are moved, once per
+ * destination rank. The R ranks are logical partitions of one GPU's buffers (or
+ * of a mapped pinned host buffer standing in for the CPU bounce buffer of
+ * Section 4.2).
+ *
+ * Conventions
+ *   - rank of expert e:  e / (E/R)     source rank of token t:  t / (T/R)
+ *   - pair order: (t,k) < (t',k')  iff  t < t' or (t == t' and k < k')
+ *   - an entry topk_idx[t][k] == -1 is masked and skipped everywhere
+ *   - receive space: one row per distinct (token, destination rank); rank r owns
+ *     rows [rank_row_offsets[r], rank_row_offsets[r+1]), ordered by token
+ *   - pair space: one entry per valid (t,k), grouped by expert id, ordered by
+ *     (t,k) inside an expert; rank r owns entries
+ *     [expert_offsets[r*E/R], expert_offsets[(r+1)*E/R])
+ *
+ * Every function returns EP_OK (0) or a negative ep_error_t. No function
+ * allocates device memory, prints, throws or aborts. Unless stated otherwise a
+ * function only enqueues work on `stream` (a cudaStream_t passed as void*; NULL
+ * is the default stream) and does not synchronise. "device" pointers must be
+ * valid on the current CUDA device; the caller owns every buffer.
+ *
+ * Shape limits, checked on the host before anything is launched
+ * (EP_ERR_INVALID_ARG otherwise): T >= 0, T % R == 0, T*K < 2^31; 1 <= K <= 32;
+ * 1 <= R <= 64; E % R == 0, R <= E <= 4096; H >= 8 and H % 8 == 0 (rows are
+ * whole 16-byte vectors); bf16 buffers 16-byte aligned.
+ */
+#ifndef EP_B200_H
+#define EP_B200_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    EP_OK = 0,
+    EP_ERR_NULL = -1,         /* a required pointer is NULL */
+    EP_ERR_INVALID_ARG = -2,  /* shape outside the limits above, misaligned buffer */
+    EP_ERR_CAPACITY = -3,     /* workspace / arena / staging buffer too small */
+    EP_ERR_CUDA = -4          /* a CUDA runtime call failed: see ep_last_cuda_error */
+} ep_error_t;
+
+/* bits of the device status word */
+#define EP_STATUS_BAD_INDEX 1 /* an expert id outside [-1, E) was seen and masked */
+#define EP_STATUS_CAPACITY  2 /* a slot >= the buffer's row capacity was skipped  */
+
+typedef struct {
+    int32_t num_tokens;  /* T */
+    int32_t top_k;       /* K */
+    int32_t hidden;      /* H, bf16 elements per row */
+    int32_t num_experts; /* E */
+    int32_t num_ranks;   /* R */
+} ep_shape_t;
+
+/* Outputs of ep_layout: device pointers to caller-allocated int32 arrays. */
+typedef struct {
+    int32_t *expert_counts;    /* [E]         valid pairs per expert                           */
+    int32_t *expert_offsets;   /* [E+1]       exclusive scan of expert_counts; [E] = P         */
+    int32_t *rank_rows;        /* [R]         distinct tokens that reach rank r                */
+    int32_t *rank_row_offsets; /* [R+1]       exclusive scan of rank_rows; [R] = N_recv        */
+    int32_t *src_row_offsets;  /* [R*(R+1)]   [r][s] = first receive row of source rank s
+                                              inside rank r; [r][R] = end of rank r           */
+    int32_t *recv_slot;        /* [T*K]       receive row of pair (t,k); -1 if masked          */
+    int32_t *pair_slot;        /* [T*K]       pair-space index of (t,k); -1 if masked          */
+    int32_t *recv_token;       /* [T*min(K,R)] receive row -> token (first N_recv entries)     */
+    int32_t *pair_row;         /* [T*K]       pair-space index -> receive row (first P)        */
+    int32_t *pair_token;       /* [T*K]       pair-space index -> token (first P)              */
+    int32_t *status;           /* [1]         EP_STATUS_* bits, rewritten by every ep_layout   */
+} ep_layout_t;
+
+/*
+ * Layout (Section 2.1: which devices a token must reach; Section 4.3: each
+ * device groups what it received by the experts it owns; Section 4.4: a
+ * receiver may start on each sender's portion separately, hence
+ * src_row_offsets). Computes every array of ep_layout_t from topk_idx
+ * [T][K] (device, int32, row-major) entirely on the device: the routing table
+ * never travels to the host (Section 4.5 names that round trip as what made
+ * routing-aware transfers slow).
+ *
+ * `workspace` (device, 16-byte aligned) must hold ep_layout_workspace_bytes()
+ * bytes; its contents need no initialisation and are garbage afterwards. Calls
+ * that share a workspace must be stream-ordered. T == 0 writes the (all-zero)
+ * counts and offsets and touches nothing else.
+ * Errors: EP_ERR_NULL, EP_ERR_INVALID_ARG, EP_ERR_CAPACITY (workspace), EP_ERR_CUDA.
+ */
+size_t ep_layout_workspace_bytes(const ep_shape_t *shape);
+int ep_layout(const ep_shape_t *shape, const int32_t *topk_idx, const ep_layout_t *out,
+              void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * Dispatch (Section 1 and Section 2.1: activations go to the devices holding the
+ * selected experts, one copy per destination device): for every valid pair
+ * recv[recv_slot[t][k]][0..H) = x[t][0..H), bit for bit. x is [T][H] bf16
+ * (device). recv is [recv_capacity_rows][H] bf16, device memory or the device
+ * alias of mapped pinned host memory. A row is written once per (token, rank).
+ * Rows no pair names are not touched. A slot >= recv_capacity_rows is skipped
+ * and sets EP_STATUS_CAPACITY in *status (device, may be NULL; bits are OR-ed
+ * in, never cleared here).
+ */
+int ep_dispatch(const ep_shape_t *shape, const void *x, const int32_t *recv_slot, void *recv,
+                int64_t recv_capacity_rows, int32_t *status, void *stream);
+
+/*
+ * Combine (Section 1; Section 4.3: the contributions that arrive for a token are
+ * added on an SM): y[t][h] = bf16( sum_k w[t][k] * out[slot[t][k]][h] ), an fp32
+ * fused multiply-add chain from +0 in ascending k, pairs with slot -1 skipped,
+ * one round-to-nearest-even narrowing at the end. out is [out_rows][H] bf16
+ * (device); slot [T][K] int32 is either pair_slot (out holds one row per pair)
+ * or recv_slot (out is a receive buffer); topk_weights [T][K] fp32; y [T][H]
+ * bf16. A slot >= out_rows is skipped and sets EP_STATUS_CAPACITY in *status
+ * (device, may be NULL).
+ */
+int ep_combine(const ep_shape_t *shape, const void *out, int64_t out_rows, const int32_t *slot,
+               const float *topk_weights, void *y, int32_t *status, void *stream);
+
+/*
+ * Local grouping by expert (Section 4.3: "groups the tokens by the experts it
+ * owns", a permutation that stays on the SMs): grouped[p] = recv[pair_row[p]]
+ * for p < P, where P is read on the device from expert_offsets[E]. grouped is
+ * [grouped_capacity_rows][H] bf16 (device); entries p >= capacity are skipped
+ * with EP_STATUS_CAPACITY.
+ */
+int ep_group(const ep_shape_t *shape, const void *recv, int64_t recv_rows, const int32_t *pair_row,
+             const int32_t *expert_offsets, void *grouped, int64_t grouped_capacity_rows,
+             int32_t *status, void *stream);
+
+/*
+ * Host-staged dispatch, copy-engine arm (Section 2.2 and Section 4.3: the DMA
+ * engines move contiguous regions only, so routing-dependent rows are first
+ * packed by a kernel): ep_dispatch into `staging` (device,
+ * [staging_capacity_rows][H]) followed by cudaMemcpyAsync device-to-host copies
+ * into recv_host (pinned host memory, same row layout) on the same stream. With
+ * rank_row_offsets_host (host, [R+1]) one copy per destination rank's partition
+ * is issued; with NULL a single copy of staging_capacity_rows rows (no row count
+ * ever reaches the host).
+ */
+int ep_dispatch_copy_engine(const ep_shape_t *shape, const void *x, const int32_t *recv_slot,
+                            const int32_t *rank_row_offsets_host, void *staging,
+                            int64_t staging_capacity_rows, void *recv_host, int32_t *status,
+                            void *stream);
+
+/*
+ * One whole step from host buffers: copies x, topk_idx and topk_weights from
+ * (pinned) host memory to the device arena, runs layout, dispatch, local
+ * grouping (the identity expert: out[p] = recv[pair_row[p]]) and combine over
+ * the pair space, and copies y back. All enqueued on `stream`; the caller
+ * synchronises. `arena` is device memory of ep_host_step_arena_bytes() bytes,
+ * 256-byte aligned. status_host (pinned host, may be NULL) receives the device
+ * status word after the step.
+ */
+size_t ep_host_step_arena_bytes(const ep_shape_t *shape);
+int ep_host_step(const ep_shape_t *shape, const void *x_host, const int32_t *topk_idx_host,
+                 const float *topk_weights_host, void *y_host, int32_t *status_host, void *arena,
+                 size_t arena_bytes, void *stream);
+
+/* Reads a device status word: copies it to *status_host and SYNCHRONISES the stream. */
+int ep_status(const int32_t *status_dev, void *stream, int32_t *status_host);
+
+/*
+ * Bandwidth probes over caller-provided buffers (no paper counterpart; they give
+ * the attainable denominators beside the nominal ones). Runs `iters` repetitions
+ * on `stream`, times each with CUDA events, SYNCHRONISES, and stores the best
+ * GB/s (10^9 bytes/s) in *gbs. kind:
+ *   EP_PROBE_READ   kernel reads `bytes` from src (device)            counts bytes
+ *   EP_PROBE_WRITE  kernel writes `bytes` to dst (device)             counts bytes
+ *   EP_PROBE_COPY   kernel copies src -> dst (device)                 counts 2*bytes
+ *   EP_PROBE_MEMCPY cudaMemcpyAsync src -> dst, any direction         counts bytes
+ * bytes must be a multiple of 16; buffers 16-byte aligned.
+ */
+#define EP_PROBE_READ   0
+#define EP_PROBE_WRITE  1
+#define EP_PROBE_COPY   2
+#define EP_PROBE_MEMCPY 3
+int ep_probe_bandwidth(int kind, void *dst, const void *src, size_t bytes, int iters, void *stream,
+                       double *gbs);
+
+/* Number of kernels this library has launched in this process (all threads). */
+int64_t ep_launch_count(void);
+
+const char *ep_strerror(int err);
+/* cudaError_t value of the most recent failed CUDA call in this process, 0 if none. */
+int ep_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* EP_B200_H */

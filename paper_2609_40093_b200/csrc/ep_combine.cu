@@ -1,0 +1,109 @@
+// ep_combine: y[t] = bf16( sum_k w[t][k] * out[slot[t][k]] ), fp32 fused multiply-add
+// chain from +0 in ascending k, one rounding to bf16 at the end.
+//
+// A group of G threads owns one token; each thread owns 16-byte columns
+// (8 bf16). For a column it first issues the loads of up to kChunk rows (they are
+// independent: this is the memory-level parallelism), then folds them into the
+// eight accumulators strictly in k order. Slots and weights sit one per lane and
+// travel by warp shuffle.
+#include "ep_common.cuh"
+
+namespace ep {
+namespace {
+
+constexpr int kBlock = 128;
+constexpr int kChunk = 8;   // rows in flight per column
+
+template <int G>
+__global__ void __launch_bounds__(kBlock)
+combine_rows_kernel(const uint4 *__restrict__ out, long long out_rows, const int32_t *__restrict__ slot,
+                    const float *__restrict__ weights, uint4 *__restrict__ y, int T, int K,
+                    int vec_per_row, int32_t *status)
+{
+    const int lane = threadIdx.x & 31;
+    const int g = threadIdx.x % G;
+    const int t = blockIdx.x * (kBlock / G) + threadIdx.x / G;
+    if (t >= T) return;                                   // whole warps leave together (G >= 32)
+
+    int32_t my_slot = -1;
+    float my_w = 0.f;
+    if (lane < K) {
+        my_slot = __ldg(slot + (size_t)t * K + lane);
+        my_w = __ldg(weights + (size_t)t * K + lane);
+        if (my_slot >= out_rows) {
+            if (status) atomicOr(status, EP_STATUS_CAPACITY);
+            my_slot = -1;
+        }
+    }
+    uint4 *dst = y + (size_t)t * vec_per_row;
+    for (int base = 0; base < vec_per_row; base += G) {   // trip count uniform over the warp
+        const int v = base + g;
+        const bool live = v < vec_per_row;
+        float acc[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) acc[i] = 0.f;
+        for (int k0 = 0; k0 < K; k0 += kChunk) {
+            uint4 row[kChunk];
+            int32_t s[kChunk];
+#pragma unroll
+            for (int j = 0; j < kChunk; ++j) {
+                s[j] = __shfl_sync(kFullMask, my_slot, (k0 + j) & 31);
+                if (k0 + j >= K) s[j] = -1;
+                if (live && s[j] >= 0) row[j] = ld_stream(out + (size_t)s[j] * vec_per_row + v);
+            }
+#pragma unroll
+            for (int j = 0; j < kChunk; ++j) {
+                const float w = __shfl_sync(kFullMask, my_w, (k0 + j) & 31);
+                if (live && s[j] >= 0) {
+                    acc[0] = __fmaf_rn(w, bf16_lo(row[j].x), acc[0]);
+                    acc[1] = __fmaf_rn(w, bf16_hi(row[j].x), acc[1]);
+                    acc[2] = __fmaf_rn(w, bf16_lo(row[j].y), acc[2]);
+                    acc[3] = __fmaf_rn(w, bf16_hi(row[j].y), acc[3]);
+                    acc[4] = __fmaf_rn(w, bf16_lo(row[j].z), acc[4]);
+                    acc[5] = __fmaf_rn(w, bf16_hi(row[j].z), acc[5]);
+                    acc[6] = __fmaf_rn(w, bf16_lo(row[j].w), acc[6]);
+                    acc[7] = __fmaf_rn(w, bf16_hi(row[j].w), acc[7]);
+                }
+            }
+        }
+        if (live) {
+            uint4 o;
+            o.x = pack_bf16x2(acc[0], acc[1]);
+            o.y = pack_bf16x2(acc[2], acc[3]);
+            o.z = pack_bf16x2(acc[4], acc[5]);
+            o.w = pack_bf16x2(acc[6], acc[7]);
+            st_stream(dst + v, o);
+        }
+    }
+}
+
+}  // namespace
+
+int launch_combine(const ep_shape_t &s, const void *out, int64_t out_rows, const int32_t *slot,
+                   const float *weights, void *y, int32_t *status, cudaStream_t stream)
+{
+    const int T = s.num_tokens, K = s.top_k, vpr = s.hidden / 8;
+    const uint4 *o = static_cast<const uint4 *>(out);
+    uint4 *yd = static_cast<uint4 *>(y);
+    if (vpr <= 64)
+        combine_rows_kernel<32><<<ceil_div(T, kBlock / 32), kBlock, 0, stream>>>(o, out_rows, slot, weights, yd, T, K, vpr, status);
+    else if (vpr <= 256)
+        combine_rows_kernel<64><<<ceil_div(T, kBlock / 64), kBlock, 0, stream>>>(o, out_rows, slot, weights, yd, T, K, vpr, status);
+    else
+        combine_rows_kernel<128><<<T, kBlock, 0, stream>>>(o, out_rows, slot, weights, yd, T, K, vpr, status);
+    EP_LAUNCH_CHECK(1);
+    return EP_OK;
+}
+
+}  // namespace ep
+
+extern "C" int ep_combine(const ep_shape_t *shape, const void *out, int64_t out_rows, const int32_t *slot,
+                          const float *topk_weights, void *y, int32_t *status, void *stream)
+{
+    int rc = ep::check_shape(shape, true);
+    if (rc != EP_OK) return rc;
+    if (shape->num_tokens == 0) return EP_OK;
+    if (!out || !slot || !topk_weights || !y) return EP_ERR_NULL;
+    if (!ep::aligned16(out) || !ep::aligned16(y) || out_rows < 0) return EP_ERR_INVALID_ARG;
+    return ep::launch_combine(*shape, out, out_rows, slot, topk_weights, y, status, static_cast<cudaStream_t>(stream));
+}

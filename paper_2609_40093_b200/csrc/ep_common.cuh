@@ -1,0 +1,95 @@
+// Shared host/device helpers of the EP library: error plumbing, shape checks,
+// 16-byte vector loads/stores with cache hints, bf16 <-> fp32 bit moves.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+#include "../../include/ep.h"
+
+namespace ep {
+
+constexpr int kMaxTopK = 32;
+constexpr int kMaxRanks = 64;
+constexpr int kMaxExperts = 4096;
+constexpr unsigned kFullMask = 0xffffffffu;
+
+// --- host side ------------------------------------------------------------
+
+void note_cuda_error(cudaError_t e);       // remembers the code for ep_last_cuda_error
+void count_launches(int n);                // feeds ep_launch_count
+
+#define EP_CUDA_TRY(expr)                                   \
+    do {                                                    \
+        cudaError_t _e = (expr);                            \
+        if (_e != cudaSuccess) {                            \
+            ::ep::note_cuda_error(_e);                      \
+            return EP_ERR_CUDA;                             \
+        }                                                   \
+    } while (0)
+
+// after a kernel launch: pick up launch-configuration errors without synchronising
+#define EP_LAUNCH_CHECK(n_launched)                         \
+    do {                                                    \
+        ::ep::count_launches(n_launched);                   \
+        EP_CUDA_TRY(cudaGetLastError());                    \
+    } while (0)
+
+inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Shape limits shared by every entry point. need_hidden: the call moves rows.
+inline int check_shape(const ep_shape_t *s, bool need_hidden)
+{
+    if (!s) return EP_ERR_NULL;
+    const int64_t T = s->num_tokens, K = s->top_k, H = s->hidden, E = s->num_experts, R = s->num_ranks;
+    if (T < 0 || K < 1 || K > kMaxTopK || R < 1 || R > kMaxRanks) return EP_ERR_INVALID_ARG;
+    if (E < R || E > kMaxExperts || E % R != 0 || T % R != 0) return EP_ERR_INVALID_ARG;
+    if (T * K >= (int64_t(1) << 31)) return EP_ERR_INVALID_ARG;
+    if (need_hidden && (H < 8 || H % 8 != 0)) return EP_ERR_INVALID_ARG;
+    return EP_OK;
+}
+
+inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+// --- device side ----------------------------------------------------------
+
+#ifdef __CUDACC__
+
+__device__ __forceinline__ unsigned lanemask_lt()
+{
+    unsigned m;
+    asm("mov.u32 %0, %%lanemask_lt;" : "=r"(m));
+    return m;
+}
+
+// Read-once 16-byte load: read-only path, do not keep the line in L1.
+__device__ __forceinline__ uint4 ld_stream(const uint4 *p)
+{
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+
+// Write-once 16-byte store (streaming: evict first).
+__device__ __forceinline__ void st_stream(uint4 *p, const uint4 &v)
+{
+    asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
+                 : "memory");
+}
+
+__device__ __forceinline__ float bf16_lo(uint32_t u) { return __uint_as_float(u << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t u) { return __uint_as_float(u & 0xffff0000u); }
+
+// two fp32 -> packed bf16x2 (lo in bits 0..15), round to nearest even
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
+{
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t *>(&v);
+}
+
+#endif  // __CUDACC__
+
+}  // namespace ep

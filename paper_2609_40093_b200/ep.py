@@ -1,0 +1,210 @@
+"""Python binding of the C-ABI CUDA library (`include/ep.h`): argument marshalling only.
+
+Every function takes torch tensors (device memory, or pinned host memory where
+the header says so), passes their addresses and the current CUDA stream to the
+library, and raises `EPError` on a non-zero return. Nothing is computed here
+and there is no fallback: if the library has not been built, the first call fails.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+
+import torch
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libep_b200.so")
+_lib = None
+
+STATUS_BAD_INDEX = 1
+STATUS_CAPACITY = 2
+PROBE_READ, PROBE_WRITE, PROBE_COPY, PROBE_MEMCPY = 0, 1, 2, 3
+
+EXPORTS = [
+    "ep_layout_workspace_bytes", "ep_layout", "ep_dispatch", "ep_combine", "ep_group",
+    "ep_dispatch_copy_engine", "ep_host_step_arena_bytes", "ep_host_step", "ep_status",
+    "ep_probe_bandwidth", "ep_launch_count", "ep_strerror", "ep_last_cuda_error",
+]
+
+
+class EPError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        msg = lib().ep_strerror(code).decode()
+        cuda = lib().ep_last_cuda_error() if code == -4 else 0
+        super().__init__(f"{where}: {msg} (code {code}" + (f", cudaError {cuda})" if cuda else ")"))
+
+
+class _Shape(ctypes.Structure):
+    _fields_ = [("num_tokens", ctypes.c_int32), ("top_k", ctypes.c_int32), ("hidden", ctypes.c_int32),
+                ("num_experts", ctypes.c_int32), ("num_ranks", ctypes.c_int32)]
+
+
+_LAYOUT_FIELDS = ["expert_counts", "expert_offsets", "rank_rows", "rank_row_offsets", "src_row_offsets",
+                  "recv_slot", "pair_slot", "recv_token", "pair_row", "pair_token", "status"]
+
+
+class _Layout(ctypes.Structure):
+    _fields_ = [(f, ctypes.c_void_p) for f in _LAYOUT_FIELDS]
+
+
+def lib() -> ctypes.CDLL:
+    """Opens the CUDA library; a missing build is an error, never a fallback."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise RuntimeError(f"{_LIB_PATH} is missing: build it with `python -m paper_2609_40093_b200.build`")
+        L = ctypes.CDLL(_LIB_PATH)
+        vp, i32, i64, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_size_t
+        sp = ctypes.POINTER(_Shape)
+        L.ep_layout_workspace_bytes.restype = sz
+        L.ep_layout_workspace_bytes.argtypes = [sp]
+        L.ep_layout.argtypes = [sp, vp, ctypes.POINTER(_Layout), vp, sz, vp]
+        L.ep_dispatch.argtypes = [sp, vp, vp, vp, i64, vp, vp]
+        L.ep_combine.argtypes = [sp, vp, i64, vp, vp, vp, vp, vp]
+        L.ep_group.argtypes = [sp, vp, i64, vp, vp, vp, i64, vp, vp]
+        L.ep_dispatch_copy_engine.argtypes = [sp, vp, vp, vp, vp, i64, vp, vp, vp]
+        L.ep_host_step_arena_bytes.restype = sz
+        L.ep_host_step_arena_bytes.argtypes = [sp]
+        L.ep_host_step.argtypes = [sp, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.ep_status.argtypes = [vp, vp, vp]
+        L.ep_probe_bandwidth.argtypes = [i32, vp, vp, sz, i32, vp, ctypes.POINTER(ctypes.c_double)]
+        L.ep_launch_count.restype = i64
+        L.ep_strerror.restype = ctypes.c_char_p
+        L.ep_strerror.argtypes = [i32]
+        for name in ["ep_layout", "ep_dispatch", "ep_combine", "ep_group", "ep_dispatch_copy_engine",
+                     "ep_host_step", "ep_status", "ep_probe_bandwidth", "ep_last_cuda_error"]:
+            getattr(L, name).restype = i32
+        _lib = L
+    return _lib
+
+
+def _shape(T, K, H, E, R) -> _Shape:
+    return _Shape(int(T), int(K), int(H), int(E), int(R))
+
+
+def _ptr(t):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream():
+    return ctypes.c_void_p(torch.cuda.current_stream().cuda_stream)
+
+
+def _check(rc: int, where: str):
+    if rc != 0:
+        raise EPError(rc, where)
+
+
+@dataclass
+class Layout:
+    """Device tensors written by `ep_layout` (all int32)."""
+    expert_counts: torch.Tensor
+    expert_offsets: torch.Tensor
+    rank_rows: torch.Tensor
+    rank_row_offsets: torch.Tensor
+    src_row_offsets: torch.Tensor
+    recv_slot: torch.Tensor
+    pair_slot: torch.Tensor
+    recv_token: torch.Tensor
+    pair_row: torch.Tensor
+    pair_token: torch.Tensor
+    status: torch.Tensor
+
+    def as_struct(self) -> _Layout:
+        return _Layout(*[getattr(self, f).data_ptr() for f in _LAYOUT_FIELDS])
+
+
+def alloc_layout(T, K, E, R, device="cuda", fill=None) -> Layout:
+    """Allocates the output arrays of `ep_layout` (torch owns the memory)."""
+    def mk(*shape):
+        n = [max(1, s) if len(shape) == 1 else s for s in shape]
+        t = torch.empty(*n, dtype=torch.int32, device=device)
+        if fill is not None:
+            t.fill_(fill)
+        return t
+    return Layout(mk(E), mk(E + 1), mk(R), mk(R + 1), mk(R, R + 1), mk(T, K), mk(T, K),
+                  mk(T * min(K, R)), mk(T * K), mk(T * K), mk(1))
+
+
+def ep_layout_workspace_bytes(T, K, E, R) -> int:
+    return int(lib().ep_layout_workspace_bytes(ctypes.byref(_shape(T, K, 8, E, R))))
+
+
+def ep_layout(topk_idx: torch.Tensor, E: int, R: int, out: Layout = None, workspace: torch.Tensor = None) -> Layout:
+    T, K = topk_idx.shape
+    if out is None:
+        out = alloc_layout(T, K, E, R, device=topk_idx.device)
+    if workspace is None:
+        workspace = torch.empty(max(16, ep_layout_workspace_bytes(T, K, E, R)), dtype=torch.uint8, device=topk_idx.device)
+    st = out.as_struct()
+    _check(lib().ep_layout(ctypes.byref(_shape(T, K, 8, E, R)), _ptr(topk_idx), ctypes.byref(st), _ptr(workspace),
+                           workspace.numel(), _stream()), "ep_layout")
+    return out
+
+
+def ep_dispatch(x: torch.Tensor, recv_slot: torch.Tensor, recv: torch.Tensor, E: int, R: int, status=None):
+    T, H = x.shape
+    K = recv_slot.shape[1]
+    _check(lib().ep_dispatch(ctypes.byref(_shape(T, K, H, E, R)), _ptr(x), _ptr(recv_slot), _ptr(recv),
+                             recv.shape[0], _ptr(status), _stream()), "ep_dispatch")
+    return recv
+
+
+def ep_combine(out: torch.Tensor, slot: torch.Tensor, topk_weights: torch.Tensor, y: torch.Tensor, E: int, R: int,
+               status=None):
+    T, K = slot.shape
+    H = out.shape[1]
+    _check(lib().ep_combine(ctypes.byref(_shape(T, K, H, E, R)), _ptr(out), out.shape[0], _ptr(slot),
+                            _ptr(topk_weights), _ptr(y), _ptr(status), _stream()), "ep_combine")
+    return y
+
+
+def ep_group(recv: torch.Tensor, lay: Layout, grouped: torch.Tensor, E: int, R: int, status=None):
+    T, K = lay.recv_slot.shape
+    H = recv.shape[1]
+    _check(lib().ep_group(ctypes.byref(_shape(T, K, H, E, R)), _ptr(recv), recv.shape[0], _ptr(lay.pair_row),
+                          _ptr(lay.expert_offsets), _ptr(grouped), grouped.shape[0], _ptr(status), _stream()),
+           "ep_group")
+    return grouped
+
+
+def ep_dispatch_copy_engine(x, recv_slot, staging, recv_host, E, R, rank_row_offsets_host=None, status=None):
+    """rank_row_offsets_host: CPU int32 tensor [R+1] or None (one worst-case copy)."""
+    T, H = x.shape
+    K = recv_slot.shape[1]
+    _check(lib().ep_dispatch_copy_engine(ctypes.byref(_shape(T, K, H, E, R)), _ptr(x), _ptr(recv_slot),
+                                         _ptr(rank_row_offsets_host), _ptr(staging), staging.shape[0],
+                                         _ptr(recv_host), _ptr(status), _stream()), "ep_dispatch_copy_engine")
+    return recv_host
+
+
+def ep_host_step_arena_bytes(T, K, H, E, R) -> int:
+    return int(lib().ep_host_step_arena_bytes(ctypes.byref(_shape(T, K, H, E, R))))
+
+
+def ep_host_step(x_host, topk_idx_host, topk_weights_host, y_host, arena, E, R, status_host=None):
+    """All *_host tensors live in (pinned) host memory; arena is a device uint8 tensor."""
+    T, H = x_host.shape
+    K = topk_idx_host.shape[1]
+    _check(lib().ep_host_step(ctypes.byref(_shape(T, K, H, E, R)), _ptr(x_host), _ptr(topk_idx_host),
+                              _ptr(topk_weights_host), _ptr(y_host), _ptr(status_host), _ptr(arena), arena.numel(),
+                              _stream()), "ep_host_step")
+    return y_host
+
+
+def ep_status(status: torch.Tensor) -> int:
+    host = ctypes.c_int32(0)
+    _check(lib().ep_status(_ptr(status), _stream(), ctypes.byref(host)), "ep_status")
+    return int(host.value)
+
+
+def ep_probe_bandwidth(kind: int, dst, src, nbytes: int, iters: int = 10) -> float:
+    g = ctypes.c_double(0.0)
+    _check(lib().ep_probe_bandwidth(kind, _ptr(dst), _ptr(src), nbytes, iters, _stream(), ctypes.byref(g)),
+           "ep_probe_bandwidth")
+    return float(g.value)
+
+
+def ep_launch_count() -> int:
+    return int(lib().ep_launch_count())

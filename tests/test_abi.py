@@ -1,0 +1,65 @@
+"""The C-ABI library loads and exports everything include/ep.h declares; host-side
+argument checks answer before anything touches a GPU."""
+import ctypes
+import os
+import re
+
+import pytest
+
+import __graft_entry__ as entry
+from paper_2609_40093_b200 import ep
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def built():
+    entry.build()
+
+
+def _declared():
+    text = open(os.path.join(ROOT, "include", "ep.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(ep_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported():
+    L = ep.lib()
+    names = _declared()
+    assert set(names) == set(ep.EXPORTS), (names, ep.EXPORTS)
+    for n in names:
+        assert getattr(L, n) is not None
+
+
+def test_host_side_validation_needs_no_gpu():
+    L = ep.lib()
+    ok = ep._shape(64, 2, 256, 8, 2)
+    assert L.ep_layout_workspace_bytes(ctypes.byref(ok)) > 0
+    assert L.ep_host_step_arena_bytes(ctypes.byref(ok)) > 64 * 256 * 2
+    bad_shapes = [
+        ep._shape(64, 0, 256, 8, 2),     # K < 1
+        ep._shape(64, 33, 256, 64, 2),   # K > 32
+        ep._shape(64, 2, 256, 9, 2),     # E % R != 0
+        ep._shape(63, 2, 256, 8, 2),     # T % R != 0
+        ep._shape(64, 2, 252, 8, 2),     # H % 8 != 0
+        ep._shape(-2, 2, 256, 8, 2),     # T < 0
+        ep._shape(64, 2, 256, 8192, 2),  # E too large
+        ep._shape(130, 2, 256, 130, 65), # R too large
+    ]
+    for s in bad_shapes:
+        assert L.ep_dispatch(ctypes.byref(s), None, None, None, 0, None, None) == -2
+        assert L.ep_layout_workspace_bytes(ctypes.byref(s)) == 0 or s.hidden == 252
+    assert L.ep_dispatch(None, None, None, None, 0, None, None) == -1
+    assert L.ep_dispatch(ctypes.byref(ok), None, None, None, 0, None, None) == -1
+    assert L.ep_combine(ctypes.byref(ok), None, 0, None, None, None, None, None) == -1
+    assert L.ep_layout(ctypes.byref(ok), None, None, None, 0, None) == -1
+    assert L.ep_dispatch(ctypes.byref(ok), ctypes.c_void_p(8), ctypes.c_void_p(16), ctypes.c_void_p(16), 4, None, None) == -2
+    assert b"NULL" in L.ep_strerror(-1) and L.ep_strerror(0) == b"ok"
+    assert L.ep_launch_count() == 0 or L.ep_launch_count() > 0
+
+
+def test_binding_refuses_to_run_without_the_library(monkeypatch, tmp_path):
+    monkeypatch.setattr(ep, "_lib", None)
+    monkeypatch.setattr(ep, "_LIB_PATH", str(tmp_path / "absent.so"))
+    with pytest.raises(RuntimeError, match="missing"):
+        ep.lib()

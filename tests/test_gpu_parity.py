@@ -1,0 +1,235 @@
+"""CUDA path vs the CPU oracle, element by element, through the C ABI.
+
+Integer outputs (layout, slots) and dispatched rows must be bit-exact. Combine must
+be within max(4e-3*|ref|, 1e-3) of the exact (fp64) sum; it is also compared bit
+for bit with the oracle's fp32 chain, which the kernel reproduces because both
+use correctly rounded fused multiply-adds in the same order.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from gpu_util import (GUARD, SENTINEL, assert_layout_equal, dev_bf16, guarded, guards_intact, host_bits,
+                      within_tolerance)
+from paper_2609_40093_b200 import ep, inputs
+
+pytestmark = pytest.mark.gpu
+
+EDGE = [  # T, H, E, K, R, routing
+    (1, 8, 1, 1, 1, "uniform"),
+    (2, 16, 2, 1, 2, "uniform"),
+    (8, 264, 8, 2, 4, "uniform"),          # H % 8 == 0 but ragged against every thread-group size
+    (96, 2880, 32, 4, 4, "uniform"),       # hidden size of a 2880-wide model: 360 vectors
+    (64, 1032, 16, 1, 8, "uniform"),       # K = 1
+    (40, 520, 16, 4, 1, "uniform"),        # R = 1
+    (48, 72, 16, 3, 16, "uniform"),        # E = R
+    (1000, 136, 512, 10, 8, "zipf"),       # 10 of 512, the finest model the paper names
+    (1056, 64, 4096, 32, 64, "uniform"),   # every maximum at once: K=32, E=4096, R=64
+    (33 * 8, 40, 24, 5, 8, "zipf_identity"),
+]
+
+
+def _run_layout(idx, E, R, fill=-7):
+    T, K = idx.shape
+    lay = ep.alloc_layout(T, K, E, R, fill=fill)
+    ep.ep_layout(torch.from_numpy(idx).cuda(), E, R, out=lay)
+    return lay
+
+
+def _full_path_check(cfg, idx, w, x, check_combine_rows=None):
+    T, K, H, E, R = cfg.T, cfg.K, cfg.H, cfg.E, cfg.R
+    ref = oracle.layout(idx, E, R)
+    lay = _run_layout(idx, E, R)
+    assert_layout_equal(lay, ref)
+    assert ep.ep_status(lay.status) == ref.status
+
+    # dispatch into a guarded buffer: rows beyond N_recv and the guards stay untouched
+    x_d = dev_bf16(x)
+    spare = 3
+    whole, recv = guarded(ref.n_recv + spare, H)
+    ep.ep_dispatch(x_d, lay.recv_slot, recv, E, R, status=lay.status)
+    got = host_bits(recv)
+    want = oracle.dispatch(x, ref.recv_slot, ref.n_recv + spare, fill=SENTINEL)
+    np.testing.assert_array_equal(got, want)
+    assert guards_intact(whole)
+
+    # local grouping: grouped[p] = recv[pair_row[p]]
+    gwhole, grouped = guarded(ref.n_pairs + spare, H)
+    ep.ep_group(recv, lay, grouped, E, R, status=lay.status)
+    gb = host_bits(grouped)
+    np.testing.assert_array_equal(gb[:ref.n_pairs], want[ref.pair_row] if ref.n_pairs else gb[:0])
+    assert (gb[ref.n_pairs:] == SENTINEL).all() and guards_intact(gwhole)
+
+    # combine over independent expert outputs in the pair space
+    out = inputs.make_out(cfg, max(1, ref.n_pairs), seed=1)
+    w_d = torch.from_numpy(w).cuda()
+    ywhole, y = guarded(T, H)
+    ep.ep_combine(dev_bf16(out), lay.pair_slot, w_d, y, E, R, status=lay.status)
+    yb = host_bits(y)
+    sel = slice(None) if check_combine_rows is None else check_combine_rows
+    y32 = oracle.combine_f32(out, ref.pair_slot[sel], w[sel])
+    y64 = oracle.combine_f64(out, ref.pair_slot[sel], w[sel])
+    assert within_tolerance(yb[sel], y64).all()
+    np.testing.assert_array_equal(yb[sel], y32)          # same fma chain => same bits
+    assert guards_intact(ywhole)
+    assert ep.ep_status(lay.status) == ref.status
+    return lay, ref
+
+
+@pytest.mark.parametrize("name", ["C1", "C2", "C3"])
+def test_configs_full_path(name):
+    cfg = inputs.CONFIGS[name]
+    d = inputs.make_inputs(cfg)
+    _full_path_check(cfg, d["topk_idx"], d["topk_weights"], d["x"])
+
+
+@pytest.mark.parametrize("T,H,E,K,R,routing", EDGE)
+def test_edge_shapes_full_path(T, H, E, K, R, routing):
+    cfg = inputs.custom_config(T, H, E, K, R, routing=routing, config_id=60)
+    d = inputs.make_inputs(cfg)
+    _full_path_check(cfg, d["topk_idx"], d["topk_weights"], d["x"])
+
+
+def test_masked_duplicate_and_bad_ids():
+    rng = np.random.default_rng(3)
+    T, H, E, K, R = 256, 128, 16, 6, 4
+    cfg = inputs.custom_config(T, H, E, K, R, config_id=61)
+    d = inputs.make_inputs(cfg)
+    idx = rng.integers(-1, E, size=(T, K)).astype(np.int32)        # duplicates inside a token, -1 masks
+    idx[5, :] = -1                                                  # a token that goes nowhere
+    idx[7, :] = 3                                                   # the same expert K times
+    lay, ref = _full_path_check(cfg, idx, d["topk_weights"], d["x"])
+    assert ref.status == 0
+    idx[11, 2] = E + 5
+    idx[200, 0] = -9
+    lay, ref = _full_path_check(cfg, idx, d["topk_weights"], d["x"])
+    assert ref.status == ep.STATUS_BAD_INDEX
+
+
+def test_all_tokens_to_one_expert_and_all_masked():
+    T, H, E, K, R = 512, 64, 8, 2, 4
+    cfg = inputs.custom_config(T, H, E, K, R, config_id=62)
+    d = inputs.make_inputs(cfg)
+    idx = np.zeros((T, K), np.int32)
+    idx[:, 1] = 1                                                   # experts 0 and 1, both on rank 0
+    _full_path_check(cfg, idx, d["topk_weights"], d["x"])
+    _full_path_check(cfg, -np.ones((T, K), np.int32), d["topk_weights"], d["x"])
+
+
+def test_empty_batch():
+    E, R, K, H = 8, 2, 2, 64
+    lay = ep.alloc_layout(0, K, E, R, fill=-7)
+    ep.ep_layout(torch.empty(0, K, dtype=torch.int32, device="cuda"), E, R, out=lay)
+    assert (lay.expert_counts.cpu() == 0).all() and (lay.rank_row_offsets.cpu() == 0).all()
+    assert (lay.expert_offsets.cpu() == 0).all() and (lay.src_row_offsets.cpu() == 0).all()
+    assert ep.ep_status(lay.status) == 0
+    x = torch.empty(0, H, dtype=torch.bfloat16, device="cuda")
+    recv = torch.empty(1, H, dtype=torch.bfloat16, device="cuda")
+    ep.ep_dispatch(x, lay.recv_slot, recv, E, R)
+    ep.ep_combine(recv, lay.recv_slot, torch.empty(0, K, device="cuda"), x, E, R)
+
+
+def test_identity_expert_roundtrip_and_one_hot_weights():
+    cfg = inputs.CONFIGS["C2"]
+    d = inputs.make_inputs(cfg)
+    idx, w, x = d["topk_idx"], d["topk_weights"], d["x"]
+    lay = _run_layout(idx, cfg.E, cfg.R)
+    n_recv = int(lay.rank_row_offsets[-1])
+    x_d = dev_bf16(x)
+    recv = torch.zeros(n_recv, cfg.H, dtype=torch.bfloat16, device="cuda")
+    ep.ep_dispatch(x_d, lay.recv_slot, recv, cfg.E, cfg.R)
+    y = torch.zeros_like(x_d)
+    ep.ep_combine(recv, lay.recv_slot, torch.from_numpy(w).cuda(), y, cfg.E, cfg.R)
+    assert within_tolerance(host_bits(y), inputs.bf16_bits_to_f32(x).astype(np.float64)).all()
+    for kstar in range(cfg.K):                                     # one-hot weights: a bit copy of the chosen row
+        onehot = torch.zeros(cfg.T, cfg.K, device="cuda")
+        onehot[:, kstar] = 1.0
+        ep.ep_combine(recv, lay.recv_slot, onehot, y, cfg.E, cfg.R)
+        np.testing.assert_array_equal(host_bits(y), x)
+
+
+def test_capacity_overflow_is_skipped_and_flagged():
+    cfg = inputs.CONFIGS["C1"]
+    d = inputs.make_inputs(cfg)
+    idx, w, x = d["topk_idx"], d["topk_weights"], d["x"]
+    ref = oracle.layout(idx, cfg.E, cfg.R)
+    lay = _run_layout(idx, cfg.E, cfg.R)
+    cap = ref.n_recv - 10
+    whole, recv = guarded(cap, cfg.H)
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ep.ep_dispatch(dev_bf16(x), lay.recv_slot, recv, cfg.E, cfg.R, status=status)
+    assert ep.ep_status(status) == ep.STATUS_CAPACITY
+    assert guards_intact(whole)
+    np.testing.assert_array_equal(host_bits(recv), oracle.dispatch(x, ref.recv_slot, ref.n_recv)[:cap])
+    # combine: slots beyond out_rows contribute nothing
+    out = inputs.make_out(cfg, ref.n_pairs)
+    status.zero_()
+    y = torch.zeros(cfg.T, cfg.H, dtype=torch.bfloat16, device="cuda")
+    short = ref.n_pairs - 7
+    ep.ep_combine(dev_bf16(out[:short]), lay.pair_slot, torch.from_numpy(w).cuda(), y, cfg.E, cfg.R, status=status)
+    assert ep.ep_status(status) == ep.STATUS_CAPACITY
+    masked = np.where(ref.pair_slot >= short, -1, ref.pair_slot).astype(np.int32)
+    np.testing.assert_array_equal(host_bits(y), oracle.combine_f32(out[:short], masked, w))
+
+
+def test_results_are_run_to_run_identical():
+    cfg = inputs.CONFIGS["C3"]
+    idx = inputs.make_topk_idx(cfg)
+    a = _run_layout(idx, cfg.E, cfg.R)
+    b = _run_layout(idx, cfg.E, cfg.R)
+    for f in ["recv_slot", "pair_slot", "recv_token", "pair_row", "pair_token"]:
+        n = int(a.rank_row_offsets[-1]) if f == "recv_token" else None
+        assert torch.equal(getattr(a, f).flatten()[:n], getattr(b, f).flatten()[:n]), f
+
+
+def test_host_step_matches_oracle():
+    cfg = inputs.CONFIGS["C3"]
+    d = inputs.make_inputs(cfg)
+    idx, w, x = d["topk_idx"], d["topk_weights"], d["x"]
+    xh = torch.from_numpy(x.view(np.int16)).view(torch.bfloat16).pin_memory()
+    ih, wh = torch.from_numpy(idx).pin_memory(), torch.from_numpy(w).pin_memory()
+    yh = torch.zeros(cfg.T, cfg.H, dtype=torch.bfloat16).pin_memory()
+    sh = torch.full((1,), -1, dtype=torch.int32).pin_memory()
+    arena = torch.empty(ep.ep_host_step_arena_bytes(cfg.T, cfg.K, cfg.H, cfg.E, cfg.R), dtype=torch.uint8, device="cuda")
+    ep.ep_host_step(xh, ih, wh, yh, arena, cfg.E, cfg.R, status_host=sh)
+    torch.cuda.synchronize()
+    assert int(sh[0]) == 0
+    ref = oracle.layout(idx, cfg.E, cfg.R)
+    recv = oracle.dispatch(x, ref.recv_slot, ref.n_recv)
+    want = oracle.combine_f32(recv[ref.pair_row], ref.pair_slot, w)
+    np.testing.assert_array_equal(yh.view(torch.int16).numpy().view(np.uint16), want)
+
+
+def test_host_staged_dispatch_both_arms():
+    """Receive buffer in mapped pinned host memory: kernel stores and the copy-engine arm."""
+    cfg = inputs.CONFIGS["C5"]
+    d = inputs.make_inputs(cfg)
+    idx, x = d["topk_idx"], d["x"]
+    ref = oracle.layout(idx, cfg.E, cfg.R)
+    want = oracle.dispatch(x, ref.recv_slot, ref.n_recv)
+    lay = _run_layout(idx, cfg.E, cfg.R)
+    x_d = dev_bf16(x)
+    # (i) the dispatch kernel stores straight into pinned host memory
+    recv_h = torch.zeros(ref.n_recv, cfg.H, dtype=torch.bfloat16).pin_memory()
+    ep.ep_dispatch(x_d, lay.recv_slot, recv_h, cfg.E, cfg.R)
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(recv_h.view(torch.int16).numpy().view(np.uint16), want)
+    # (ii) pack on the device, then one copy-engine transfer per destination rank
+    staging = torch.zeros(ref.n_recv, cfg.H, dtype=torch.bfloat16, device="cuda")
+    for offsets in (lay.rank_row_offsets.cpu(), None):
+        recv_h.zero_()
+        ep.ep_dispatch_copy_engine(x_d, lay.recv_slot, staging, recv_h, cfg.E, cfg.R, rank_row_offsets_host=offsets)
+        torch.cuda.synchronize()
+        np.testing.assert_array_equal(recv_h.view(torch.int16).numpy().view(np.uint16), want)
+
+
+def test_largest_config_sampled():
+    """C4 in the launch configuration the benchmark times: integer outputs and the
+    dispatched buffer in full, combine on sampled tokens."""
+    cfg = inputs.CONFIGS["C4"]
+    d = inputs.make_inputs(cfg)
+    idx, w, x = d["topk_idx"], d["topk_weights"], d["x"]
+    rows = np.random.default_rng(0).choice(cfg.T, size=192, replace=False)
+    rows.sort()
+    _full_path_check(cfg, idx, w, x, check_combine_rows=rows)
