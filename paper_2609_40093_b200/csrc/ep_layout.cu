@@ -279,8 +279,10 @@ extern "C" int ep_layout(const ep_shape_t *shape, const int32_t *topk_idx, const
     if (rc != EP_OK) return rc;
     if (!out || !workspace) return EP_ERR_NULL;
     if (!out->expert_counts || !out->expert_offsets || !out->rank_rows || !out->rank_row_offsets ||
-        !out->src_row_offsets || !out->recv_slot || !out->pair_slot || !out->recv_token ||
-        !out->pair_row || !out->pair_token || !out->status)
+        !out->src_row_offsets || !out->status)
+        return EP_ERR_NULL;
+    if (shape->num_tokens > 0 && (!out->recv_slot || !out->pair_slot || !out->recv_token || !out->pair_row ||
+                                  !out->pair_token))
         return EP_ERR_NULL;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     const LayoutPlan plan = make_plan(*shape);

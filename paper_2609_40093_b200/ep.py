@@ -118,11 +118,13 @@ class Layout:
 def alloc_layout(T, K, E, R, device="cuda", fill=None) -> Layout:
     """Allocates the output arrays of `ep_layout` (torch owns the memory)."""
     def mk(*shape):
-        n = [max(1, s) if len(shape) == 1 else s for s in shape]
-        t = torch.empty(*n, dtype=torch.int32, device=device)
+        n = 1
+        for d in shape:
+            n *= d
+        t = torch.empty(max(1, n), dtype=torch.int32, device=device)   # never a NULL pointer, even for T == 0
         if fill is not None:
             t.fill_(fill)
-        return t
+        return t[:n].view(*shape)
     return Layout(mk(E), mk(E + 1), mk(R), mk(R + 1), mk(R, R + 1), mk(T, K), mk(T, K),
                   mk(T * min(K, R)), mk(T * K), mk(T * K), mk(1))
 

@@ -19,8 +19,7 @@ def host_bits(t: torch.Tensor) -> np.ndarray:
 
 def guarded(rows: int, H: int):
     """A [rows+2*GUARD, H] bf16 device buffer full of the sentinel; returns (whole, view of the middle)."""
-    whole = torch.full((rows + 2 * GUARD, H), SENTINEL, dtype=torch.int16 if SENTINEL < 0x8000 else torch.int32,
-                       device="cuda").to(torch.int16).view(torch.bfloat16)
+    whole = torch.full((rows + 2 * GUARD, H), SENTINEL, dtype=torch.int16, device="cuda").view(torch.bfloat16)
     return whole, whole[GUARD:GUARD + rows]
 
 
