@@ -51,7 +51,8 @@ typedef enum {
     EP_ERR_NULL = -1,         /* a required pointer is NULL */
     EP_ERR_INVALID_ARG = -2,  /* shape outside the limits above, misaligned buffer */
     EP_ERR_CAPACITY = -3,     /* workspace / arena / staging buffer too small */
-    EP_ERR_CUDA = -4          /* a CUDA runtime call failed: see ep_last_cuda_error */
+    EP_ERR_CUDA = -4,         /* a CUDA runtime call failed: see ep_last_cuda_error */
+    EP_ERR_STATIC_SCRATCH = -5 /* ep_layout_static: the shape needs more scratch than the fixed array holds */
 } ep_error_t;
 
 /* bits of the device status word */
@@ -100,6 +101,36 @@ typedef struct {
 size_t ep_layout_workspace_bytes(const ep_shape_t *shape);
 int ep_layout(const ep_shape_t *shape, const int32_t *topk_idx, const ep_layout_t *out,
               void *workspace, size_t workspace_bytes, void *stream);
+
+/*
+ * Layout without any allocation (the paper has no counterpart; this entry point
+ * exists for integration reasons only). Some callers cannot obtain device
+ * memory at the point where they need a layout: code running inside a serving
+ * engine whose memory pool is fully handed out, a plugin that is forbidden to
+ * call cudaMalloc, a component that must not disturb a caching allocator. For
+ * them this call computes exactly what ep_layout computes -- same arguments
+ * minus the workspace, same outputs bit for bit, same errors -- but takes its
+ * scratch from a fixed array of EP_LAYOUT_STATIC_SCRATCH_BYTES bytes that lives
+ * inside the library on every GPU that loads it, until the process exits. It
+ * calls no cudaMalloc, cudaFree or other allocating routine. The caller still
+ * provides topk_idx and every output array.
+ *
+ *   - Limit: the scratch a shape needs is ep_layout_workspace_bytes(shape)
+ *     (about 4*(E+R+1) bytes per 32 tokens up to 32768 tokens, constant beyond);
+ *     shapes that need more than the array holds return EP_ERR_STATIC_SCRATCH
+ *     and enqueue nothing. The five benchmark configurations all fit.
+ *   - First call on a device: looks up the array's device address (once per
+ *     device, with that device current). Make that first call outside any
+ *     stream capture.
+ *   - The array is shared by every call on that device and keeps what the last
+ *     call left in it; the kernels rewrite all they read, so no clearing is
+ *     needed. Two calls that overlap on the GPU (different streams, no ordering)
+ *     race on it: order them.
+ */
+#define EP_LAYOUT_STATIC_SCRATCH_BYTES (1u << 20)
+size_t ep_layout_static_scratch_bytes(void);
+int ep_layout_static(const ep_shape_t *shape, const int32_t *topk_idx, const ep_layout_t *out,
+                     void *stream);
 
 /*
  * Dispatch (Section 1 and Section 2.1: activations go to the devices holding the

@@ -257,6 +257,9 @@ extern "C" const char *ep_strerror(int err)
     case EP_ERR_INVALID_ARG: return "invalid argument (shape outside the supported limits or misaligned buffer)";
     case EP_ERR_CAPACITY: return "a caller-provided buffer is too small";
     case EP_ERR_CUDA: return "a CUDA runtime call failed (see ep_last_cuda_error)";
+    case EP_ERR_STATIC_SCRATCH:
+        return "ep_layout_static: this shape needs more scratch than the library's fixed array holds; "
+               "use ep_layout with a caller-provided workspace";
     default: return "unknown error";
     }
 }

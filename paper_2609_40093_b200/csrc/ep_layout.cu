@@ -16,6 +16,8 @@
 //                                                    -> slots and inverse maps
 //
 // Bins: [0,E) experts, [E,E+R) rank hits, [E+R] ids outside [-1,E).
+#include <mutex>
+
 #include "ep_common.cuh"
 
 namespace ep {
@@ -323,4 +325,56 @@ extern "C" int ep_layout(const ep_shape_t *shape, const int32_t *topk_idx, const
     layout_assign_kernel<<<grid_tiles, plan.warps * 32, plan.smem_assign, stream>>>(a);
     EP_LAUNCH_CHECK(3);
     return EP_OK;
+}
+
+// ---------------------------------------------------------------------------
+// ep_layout_static: the same layout with its scratch in a fixed device array, for
+// callers that are not allowed to allocate device memory.
+namespace ep {
+namespace {
+
+// Scratch of the allocation-free entry point. Every GPU on which this library is
+// loaded holds these bytes until the process exits. In host code this name is
+// only a handle: the device address comes from cudaGetSymbolAddress below.
+static __device__ __align__(256) unsigned char g_layout_static_scratch[EP_LAYOUT_STATIC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+void *g_static_scratch_ptr[kMaxDevices] = {};      // device address of the array, per device
+std::mutex g_static_scratch_mutex;
+
+// Looks the array's device address up once per device, with that device current.
+int static_scratch_address(void **ptr)
+{
+    int dev = -1;
+    EP_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= kMaxDevices) return EP_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lock(g_static_scratch_mutex);
+    if (!g_static_scratch_ptr[dev]) {
+        void *p = nullptr;
+        EP_CUDA_TRY(cudaGetSymbolAddress(&p, g_layout_static_scratch));
+        if (!p) return EP_ERR_CUDA;
+        g_static_scratch_ptr[dev] = p;
+    }
+    *ptr = g_static_scratch_ptr[dev];
+    return EP_OK;
+}
+
+}  // namespace
+}  // namespace ep
+
+extern "C" size_t ep_layout_static_scratch_bytes(void) { return EP_LAYOUT_STATIC_SCRATCH_BYTES; }
+
+extern "C" int ep_layout_static(const ep_shape_t *shape, const int32_t *topk_idx, const ep_layout_t *out,
+                                void *stream)
+{
+    int rc = ep::check_shape(shape, false);
+    if (rc != EP_OK) return rc;
+    // shapes whose scratch does not fit the fixed array are refused before anything is enqueued
+    if (ep::make_plan(*shape).workspace_bytes > (size_t)EP_LAYOUT_STATIC_SCRATCH_BYTES) return EP_ERR_STATIC_SCRATCH;
+    void *scratch = nullptr;
+    rc = ep::static_scratch_address(&scratch);
+    if (rc != EP_OK) return rc;
+    // pass 1 rewrites every scratch word it later reads (including the CTA ticket),
+    // so whatever the previous call left in the array needs no clearing
+    return ep_layout(shape, topk_idx, out, scratch, EP_LAYOUT_STATIC_SCRATCH_BYTES, stream);
 }

@@ -21,7 +21,7 @@ STATUS_CAPACITY = 2
 PROBE_READ, PROBE_WRITE, PROBE_COPY, PROBE_MEMCPY = 0, 1, 2, 3
 
 EXPORTS = [
-    "ep_layout_workspace_bytes", "ep_layout", "ep_dispatch", "ep_combine", "ep_group",
+    "ep_layout_workspace_bytes", "ep_layout", "ep_layout_static", "ep_layout_static_scratch_bytes", "ep_dispatch", "ep_combine", "ep_group",
     "ep_dispatch_copy_engine", "ep_host_step_arena_bytes", "ep_host_step", "ep_status",
     "ep_probe_bandwidth", "ep_launch_count", "ep_strerror", "ep_last_cuda_error",
 ]
@@ -60,6 +60,9 @@ def lib() -> ctypes.CDLL:
         L.ep_layout_workspace_bytes.restype = sz
         L.ep_layout_workspace_bytes.argtypes = [sp]
         L.ep_layout.argtypes = [sp, vp, ctypes.POINTER(_Layout), vp, sz, vp]
+        L.ep_layout_static.argtypes = [sp, vp, ctypes.POINTER(_Layout), vp]
+        L.ep_layout_static.restype = i32
+        L.ep_layout_static_scratch_bytes.restype = sz
         L.ep_dispatch.argtypes = [sp, vp, vp, vp, i64, vp, vp]
         L.ep_combine.argtypes = [sp, vp, i64, vp, vp, vp, vp, vp]
         L.ep_group.argtypes = [sp, vp, i64, vp, vp, vp, i64, vp, vp]
@@ -143,6 +146,21 @@ def ep_layout(topk_idx: torch.Tensor, E: int, R: int, out: Layout = None, worksp
     _check(lib().ep_layout(ctypes.byref(_shape(T, K, 8, E, R)), _ptr(topk_idx), ctypes.byref(st), _ptr(workspace),
                            workspace.numel(), _stream()), "ep_layout")
     return out
+
+
+def ep_layout_static(topk_idx: torch.Tensor, E: int, R: int, out: Layout) -> Layout:
+    """`ep_layout` for callers that may not allocate device memory: the scratch is a
+    fixed array inside the library, so `out` must be given and nothing is allocated
+    here either. Shapes whose scratch exceeds `ep_layout_static_scratch_bytes()` raise."""
+    T, K = topk_idx.shape
+    st = out.as_struct()
+    _check(lib().ep_layout_static(ctypes.byref(_shape(T, K, 8, E, R)), _ptr(topk_idx), ctypes.byref(st), _stream()),
+           "ep_layout_static")
+    return out
+
+
+def ep_layout_static_scratch_bytes() -> int:
+    return int(lib().ep_layout_static_scratch_bytes())
 
 
 def ep_dispatch(x: torch.Tensor, recv_slot: torch.Tensor, recv: torch.Tensor, E: int, R: int, status=None):
