@@ -344,7 +344,7 @@ def main():
                    "l2": "working set per step exceeds L2 (no flush needed)" if alg["combine"] > 2 * 126e6
                    else "working set fits L2: warm-L2 latency figures", "n_recv": n_recv, "n_pairs": n_pairs},
         "ops": {
-            "layout": {"us": lay_ms * 1e3, "launches_per_step": 3},
+            "layout": {"us": lay_ms * 1e3},
             "dispatch": {"us": dis_ms * 1e3, "GB/s": dis_gbs, "tokens/s": T / (dis_ms * 1e-3), "bytes": alg["dispatch"]},
             "combine": {"us": com_ms * 1e3, "GB/s": com_gbs, "tokens/s": T / (com_ms * 1e-3), "bytes": alg["combine"]},
         },

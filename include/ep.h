@@ -115,10 +115,11 @@ int ep_layout(const ep_shape_t *shape, const int32_t *topk_idx, const ep_layout_
  * calls no cudaMalloc, cudaFree or other allocating routine. The caller still
  * provides topk_idx and every output array.
  *
- *   - Limit: the scratch a shape needs is ep_layout_workspace_bytes(shape)
- *     (about 4*(E+R+1) bytes per 32 tokens up to 32768 tokens, constant beyond);
- *     shapes that need more than the array holds return EP_ERR_STATIC_SCRATCH
- *     and enqueue nothing. The five benchmark configurations all fit.
+ *   - Limit: the scratch a shape needs is ep_layout_workspace_bytes(shape): 16
+ *     bytes for batches of up to 2048 tokens, else 4*(E+R+1) bytes per CTA of
+ *     8 token tiles, at most 128 CTAs (34 KB for T=8192, E=256, R=8). Shapes
+ *     that need more than the array holds return EP_ERR_STATIC_SCRATCH and
+ *     enqueue nothing.
  *   - First call on a device: looks up the array's device address (once per
  *     device, with that device current). Make that first call outside any
  *     stream capture.

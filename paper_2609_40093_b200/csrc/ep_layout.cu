@@ -2,227 +2,337 @@
 //
 // The work is a stable counting sort of the T*K (token, k) pairs by expert id plus
 // a stable count of the distinct (token, rank) hits. Determinism never depends on
-// the arrival order of atomics: tokens are cut into contiguous tiles, one warp
-// owns a tile, and every rank inside a tile is derived from warp ballots /
-// matches whose lane order is the (t,k) order.
-//
-//   pass 1  count   one warp per tile: histogram of experts, of rank hits and of
-//                   bad ids over the tile            -> part[tile][bin]
-//   pass 2  scan    one warp per bin: exclusive scan of part[.][bin] over tiles
-//                   (in place) and the bin total; the last CTA to finish scans
-//                   the totals over bins             -> counts, offsets, status
-//   pass 3  assign  one warp per tile: replays the tile in order with running
-//                   counters that start at offset[bin] + part[tile][bin]
-//                                                    -> slots and inverse maps
-//
+// the arrival order of atomics: tokens are cut into contiguous tiles of 32*m
+// tokens, one warp owns a tile, a CTA owns `warps` consecutive tiles, and every
+// rank inside a tile comes from warp ballots / matches whose lane order is the
+// (t,k) order. Every CTA
+//   1. histograms its tiles (experts, rank hits, bad ids) in shared memory,
+//   2. learns, per bin, the count in earlier CTAs and the grand total,
+//   3. scans the totals over bins (expert_offsets, rank_row_offsets),
+//   4. replays its tiles in (t,k) order with running counters that start at
+//      offset[bin] + earlier CTAs + earlier warps of this CTA.
+// Step 2 has three forms:
+//   single   one CTA holds every tile: nothing to exchange;
+//   cluster  up to 8 CTAs form one thread-block cluster and read each other's CTA
+//            totals through distributed shared memory between two cluster barriers:
+//            one launch, no global scratch (all five benchmark shapes take this path);
+//   global   larger batches: a first kernel writes cta_part[cta][bin] to the
+//            workspace; the main kernel, launched with programmatic stream
+//            serialisation so that its histogram phase overlaps the first kernel,
+//            executes griddepcontrol.wait and then reads every cta_part row.
 // Bins: [0,E) experts, [E,E+R) rank hits, [E+R] ids outside [-1,E).
+#include <cooperative_groups.h>
+
 #include <mutex>
 
 #include "ep_common.cuh"
 
+namespace cg = cooperative_groups;
+
 namespace ep {
 namespace {
 
-constexpr int kMaxTiles = 1024;     // lanes of the scan warp own <= 32 tiles each
-constexpr int kScanWarps = 4;
+constexpr int kMaxWarpsSingle = 32;     // one CTA holds every tile: up to 1024 tokens
+constexpr int kMaxWarps = 8;            // tiles per CTA otherwise (the replay is throughput-bound per SM: spread it)
+constexpr int kMaxCluster = 8;          // portable cluster size
+constexpr int kMaxCtasGlobal = 128;
+constexpr size_t kSmemBudget = 200 * 1024;
+
+enum { kModeSingle = 0, kModeCluster = 1, kModeGlobal = 2 };
 
 struct LayoutPlan {
+    int mode;
     int tile_tokens;    // tokens per tile, a multiple of 32
     int n_tiles;
     int bins;           // E + R + 1
-    int warps;          // warps (tiles) per CTA in pass 1 and 3
-    size_t smem_count;  // dynamic shared memory, pass 1
-    size_t smem_assign; // dynamic shared memory, pass 3
+    int warps;          // tiles per CTA
+    int n_ctas;
+    size_t smem;        // dynamic shared memory
     size_t workspace_bytes;
 };
+
+// shared memory: per warp  hist[bins] | ballots[kMaxRanks] | slots[32*K] | ids[32*K];
+//                per CTA   tot_e[E+1] | tot_r[R+1] | pre[bins] | cta_tot[bins] | scan[32]
+inline size_t per_warp_ints(int bins, int K) { return (size_t)bins + kMaxRanks + 64 * (size_t)K; }
+inline size_t per_cta_ints(int bins) { return 3 * (size_t)bins + 2 + 32; }
 
 LayoutPlan make_plan(const ep_shape_t &s)
 {
     LayoutPlan p;
-    const int T = s.num_tokens;
-    int per = ceil_div(ceil_div(T > 0 ? T : 1, kMaxTiles), 32) * 32;
-    p.tile_tokens = per < 32 ? 32 : per;
-    p.n_tiles = ceil_div(T, p.tile_tokens);
+    const int T = s.num_tokens > 0 ? s.num_tokens : 1;
     p.bins = s.num_experts + s.num_ranks + 1;
-    // per-warp shared memory of pass 3: running counters + ballots + staged receive slots
-    size_t per_warp = sizeof(int32_t) * (size_t)(p.bins + kMaxRanks + 32 * s.top_k);
-    int w = (int)((96 * 1024) / per_warp);
-    p.warps = w < 1 ? 1 : (w > 8 ? 8 : w);
-    p.smem_assign = per_warp * p.warps;
-    p.smem_count = sizeof(int32_t) * (size_t)p.bins * p.warps;
-    p.workspace_bytes = sizeof(int32_t) * ((size_t)(p.n_tiles > 0 ? p.n_tiles : 1) * p.bins + p.bins + 4);
+    const size_t pw = sizeof(int32_t) * per_warp_ints(p.bins, s.top_k), pc = sizeof(int32_t) * per_cta_ints(p.bins);
+    int fit = (int)((kSmemBudget - pc) / pw);
+    fit = fit < 1 ? 1 : fit;
+    const int groups = ceil_div(T, 32);                 // 32-token groups
+    const int w1 = fit > kMaxWarpsSingle ? kMaxWarpsSingle : fit;
+    const int w = fit > kMaxWarps ? kMaxWarps : fit;
+    if (groups <= w1) {
+        p.mode = kModeSingle;
+        p.tile_tokens = 32;
+        p.n_tiles = groups;
+        p.warps = groups;
+        p.n_ctas = 1;
+    } else {
+        p.tile_tokens = 32 * ceil_div(groups, kMaxCtasGlobal * w);
+        p.n_tiles = ceil_div(T, p.tile_tokens);
+        p.warps = w;
+        p.n_ctas = ceil_div(p.n_tiles, w);
+        p.mode = p.n_ctas <= kMaxCluster ? kModeCluster : kModeGlobal;
+    }
+    p.smem = pw * p.warps + pc;
+    p.workspace_bytes = p.mode == kModeGlobal ? sizeof(int32_t) * (size_t)p.n_ctas * p.bins : 16;
     return p;
 }
 
+// n / d for 0 <= n < 2^31 by one 64x64 high multiply: m = ceil(2^64 / d)
+struct FastDiv {
+    uint32_t d;
+    uint64_t m;
+};
+inline FastDiv make_fastdiv(int d)
+{
+    FastDiv f;
+    f.d = (uint32_t)d;
+    f.m = d > 1 ? ~uint64_t(0) / (uint64_t)d + 1 : 0;
+    return f;
+}
+__device__ __forceinline__ int fdiv(int n, const FastDiv &f)
+{
+    return f.d == 1 ? n : (int)__umul64hi((uint64_t)(uint32_t)n, f.m);
+}
+
+// phase time stamps of the main kernel, compiled only with -DEP_LAYOUT_TIMING (never in the product build)
+#ifdef EP_LAYOUT_TIMING
+static long long *g_timing_buf = nullptr;
+#define EP_STAMP(i) do { if (a.dbg && threadIdx.x == 0) a.dbg[blockIdx.x * 16 + (i)] = clock64(); } while (0)
+#else
+#define EP_STAMP(i) do { } while (0)
+#endif
+
 struct LayoutArgs {
+#ifdef EP_LAYOUT_TIMING
+    long long *dbg;
+#endif
     const int32_t *idx;
     ep_layout_t out;
-    int32_t *part;      // [n_tiles][bins]
-    int32_t *totals;    // [bins]
-    unsigned *ticket;   // [1]
-    int T, K, E, R, El, Tr;
-    int tile_tokens, n_tiles, bins;
+    int32_t *cta_part;  // [n_ctas][bins], global form only
+    int T, K, E, R, Tr;
+    FastDiv by_El, by_K, by_Tr;
+    int tile_tokens, n_tiles, bins, n_ctas, mode;
 };
 
-// ---------------------------------------------------------------- pass 1
-__global__ void layout_count_kernel(LayoutArgs a)
+// The warp copies the expert ids of the 32 tokens [tb, tb+32) into ids[32*K] (coalesced, all loads in
+// flight at once); entries of tokens >= t1 become -1. Returns the number of live items.
+__device__ __forceinline__ int stage_group(const LayoutArgs &a, int32_t *ids, int tb, int t1, int lane)
 {
-    extern __shared__ int32_t smem[];
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int tile = blockIdx.x * (blockDim.x >> 5) + warp;
-    if (blockIdx.x == 0 && threadIdx.x == 0) *a.ticket = 0u;     // pass 2 counts finished CTAs here
-    if (tile >= a.n_tiles) return;
-    int32_t *hist = smem + warp * a.bins;
+    const int n_items = (min(t1, tb + 32) - tb) * a.K;
+    const int32_t *src = a.idx + (size_t)tb * a.K;
+    for (int i = lane; i < 32 * a.K; i += 32) ids[i] = i < n_items ? __ldg(src + i) : -1;
+    __syncwarp();
+    return n_items;
+}
+
+// rank bitmask of the token this lane owns in the staged group
+__device__ __forceinline__ unsigned long long token_rank_mask(const LayoutArgs &a, const int32_t *ids, int lane)
+{
+    unsigned long long mask = 0ull;
+    for (int k = 0; k < a.K; ++k) {
+        const int e = ids[lane * a.K + k];
+        if (e >= 0 && e < a.E) mask |= 1ull << fdiv(e, a.by_El);
+    }
+    return mask;
+}
+
+// One warp counts its tile into hist[bins] (shared memory, this warp's own).
+__device__ __forceinline__ void count_tile(const LayoutArgs &a, int32_t *hist, int32_t *ids, int tile, int lane)
+{
     for (int b = lane; b < a.bins; b += 32) hist[b] = 0;
     __syncwarp();
-
+    if (tile >= a.n_tiles) return;
     const int t0 = tile * a.tile_tokens;
     const int t1 = min(a.T, t0 + a.tile_tokens);
-    // experts: any order
     int bad = 0;
-    for (int i = t0 * a.K + lane; i < t1 * a.K; i += 32) {
-        const int e = __ldg(a.idx + i);
-        if (e >= 0 && e < a.E) atomicAdd(hist + e, 1);
-        else if (e != -1) ++bad;
-    }
-    if (bad) atomicAdd(hist + a.E + a.R, bad);
-    // rank hits: one token per lane, one ballot per rank
     for (int tb = t0; tb < t1; tb += 32) {
-        const int t = tb + lane;
-        unsigned long long mask = 0ull;
-        if (t < t1)
-            for (int k = 0; k < a.K; ++k) {
-                const int e = __ldg(a.idx + (size_t)t * a.K + k);
-                if (e >= 0 && e < a.E) mask |= 1ull << (e / a.El);
-            }
+        const int n_items = stage_group(a, ids, tb, t1, lane);
+        for (int i = lane; i < n_items; i += 32) {                   // experts: any order
+            const int e = ids[i];
+            if (e >= 0 && e < a.E) atomicAdd(hist + e, 1);
+            else if (e != -1) ++bad;
+        }
+        const unsigned long long mask = token_rank_mask(a, ids, lane);   // rank hits: token per lane, ballot per rank
         for (int r = 0; r < a.R; ++r) {
             const unsigned b = __ballot_sync(kFullMask, (mask >> r) & 1ull);
             if (lane == 0) hist[a.E + r] += __popc(b);
         }
+        __syncwarp();
     }
+    if (bad) atomicAdd(hist + a.E + a.R, bad);
     __syncwarp();
-    int32_t *dst = a.part + (size_t)tile * a.bins;
-    for (int b = lane; b < a.bins; b += 32) dst[b] = hist[b];
 }
 
-// ---------------------------------------------------------------- pass 2
-// exclusive scan of in[0..n) into out[0..n], out[n] = total; whole CTA, n <= 4096+
-__device__ void block_exclusive_scan(const int32_t *in, int32_t *out, int n, int32_t *sh /* [blockDim.x] */)
+// exclusive scan of v[0..n) in place (shared memory), v[n] = total; whole CTA; sh holds one int per warp
+__device__ void block_exclusive_scan_smem(int32_t *v, int n, int32_t *sh)
 {
-    const int nt = blockDim.x, tid = threadIdx.x;
+    const int nt = blockDim.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nw = nt >> 5;
     const int chunk = (n + nt - 1) / nt;
     const int lo = min(n, tid * chunk), hi = min(n, lo + chunk);
     int32_t sum = 0;
-    for (int i = lo; i < hi; ++i) sum += __ldcg(in + i);     // written by other CTAs: read at L2
-    sh[tid] = sum;
-    __syncthreads();
-    for (int off = 1; off < nt; off <<= 1) {      // Hillis-Steele inclusive scan over the chunk sums
-        int32_t v = tid >= off ? sh[tid - off] : 0;
-        __syncthreads();
-        sh[tid] += v;
-        __syncthreads();
+    for (int i = lo; i < hi; ++i) sum += v[i];
+    int32_t incl = sum;                              // inclusive scan of the chunk sums inside the warp
+    for (int off = 1; off < 32; off <<= 1) {
+        const int32_t up = __shfl_up_sync(kFullMask, incl, off);
+        if (lane >= off) incl += up;
     }
-    int32_t run = sh[tid] - sum;
-    for (int i = lo; i < hi; ++i) {
-        const int32_t v = __ldcg(in + i);
-        out[i] = run;
-        run += v;
-    }
-    if (tid == nt - 1) out[n] = sh[tid];
+    if (lane == 31) sh[warp] = incl;
     __syncthreads();
-}
-
-__global__ void layout_scan_kernel(LayoutArgs a)
-{
-    __shared__ int32_t sh[kScanWarps * 32];
-    __shared__ bool is_last;
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int bin = blockIdx.x * kScanWarps + warp;
-    if (bin < a.bins) {
-        const int c = (a.n_tiles + 31) >> 5;                   // tiles owned by a lane, contiguous
-        const int lo = min(a.n_tiles, lane * c), hi = min(a.n_tiles, lo + c);
-        int32_t sum = 0;
-        for (int j = lo; j < hi; ++j) sum += a.part[(size_t)j * a.bins + bin];
-        int32_t incl = sum;
+    if (warp == 0) {                                 // exclusive scan of the warp totals
+        const int32_t w = lane < nw ? sh[lane] : 0;
+        int32_t wi = w;
         for (int off = 1; off < 32; off <<= 1) {
-            const int32_t v = __shfl_up_sync(kFullMask, incl, off);
-            if (lane >= off) incl += v;
+            const int32_t up = __shfl_up_sync(kFullMask, wi, off);
+            if (lane >= off) wi += up;
         }
-        int32_t run = incl - sum;
-        for (int j = lo; j < hi; ++j) {
-            int32_t *p = a.part + (size_t)j * a.bins + bin;
-            const int32_t v = *p;
-            *p = run;
-            run += v;
-        }
-        if (lane == 31) {
-            a.totals[bin] = incl;
-            if (bin < a.E) a.out.expert_counts[bin] = incl;
-            else if (bin < a.E + a.R) a.out.rank_rows[bin - a.E] = incl;
-        }
+        if (lane < nw) sh[lane] = wi - w;
     }
-    // the last CTA to get here scans the totals over the bins
-    __threadfence();
     __syncthreads();
-    if (threadIdx.x == 0) is_last = (atomicAdd(a.ticket, 1u) == gridDim.x - 1);
+    int32_t run = sh[warp] + incl - sum;
+    for (int i = lo; i < hi; ++i) {
+        const int32_t x = v[i];
+        v[i] = run;
+        run += x;
+    }
+    if (tid == nt - 1) v[n] = run;
     __syncthreads();
-    if (!is_last) return;
-    __threadfence();
-    block_exclusive_scan(a.totals, a.out.expert_offsets, a.E, sh);
-    block_exclusive_scan(a.totals + a.E, a.out.rank_row_offsets, a.R, sh);
-    for (int r = threadIdx.x; r < a.R; r += blockDim.x)
-        a.out.src_row_offsets[r * (a.R + 1) + a.R] = a.out.rank_row_offsets[r + 1];
-    if (threadIdx.x == 0) *a.out.status = __ldcg(a.totals + a.E + a.R) ? EP_STATUS_BAD_INDEX : 0;
 }
 
-// ---------------------------------------------------------------- pass 3
-__global__ void layout_assign_kernel(LayoutArgs a)
+// ---------------------------------------------------------------- global form, first kernel
+__global__ void __launch_bounds__(kMaxWarps * 32) layout_cta_count_kernel(LayoutArgs a)
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the main kernel may start its own counting now
+    extern __shared__ int32_t smem[];
+    const int warps = blockDim.x >> 5, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int pw = a.bins + kMaxRanks + 64 * a.K;
+    count_tile(a, smem + warp * pw, smem + warp * pw + a.bins + kMaxRanks + 32 * a.K, blockIdx.x * warps + warp, lane);
+    __syncthreads();
+    int32_t *dst = a.cta_part + (size_t)blockIdx.x * a.bins;
+    for (int b = threadIdx.x; b < a.bins; b += blockDim.x) {
+        int32_t sum = 0;
+        for (int w = 0; w < warps; ++w) sum += smem[w * pw + b];
+        dst[b] = sum;
+    }
+}
+
+// ---------------------------------------------------------------- main kernel
+__global__ void __launch_bounds__(kMaxWarpsSingle * 32) layout_assign_kernel(LayoutArgs a)
 {
     extern __shared__ int32_t smem[];
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int tile = blockIdx.x * (blockDim.x >> 5) + warp;
-    if (tile >= a.n_tiles) return;
+    const int warps = blockDim.x >> 5, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int pw = a.bins + kMaxRanks + 64 * a.K;
     const int nb = a.E + a.R;
-    const int per_warp = a.bins + kMaxRanks + 32 * a.K;
-    int32_t *run = smem + warp * per_warp;           // [E+R] next free slot of each bin
-    unsigned *bal = reinterpret_cast<unsigned *>(run + a.bins);   // [R] ballot of the current 32 tokens
-    int32_t *slot_s = run + a.bins + kMaxRanks;      // [32*K] receive slots of the current 32 tokens
+    int32_t *run = smem + warp * pw;                                 // [bins] histogram, later next free slot
+    unsigned *bal = reinterpret_cast<unsigned *>(run + a.bins);      // [R] ballots of the current 32 tokens
+    int32_t *slot_s = run + a.bins + kMaxRanks;                      // [32*K] receive slots of the current 32 tokens
+    int32_t *ids = slot_s + 32 * a.K;                                // [32*K] expert ids of the current 32 tokens
+    int32_t *tot_e = smem + warps * pw;                              // [E+1] expert totals -> offsets
+    int32_t *tot_r = tot_e + a.E + 1;                                // [R+1] rank totals -> offsets
+    int32_t *pre = tot_r + a.R + 1;                                  // [bins] count in earlier CTAs
+    int32_t *cta_tot = pre + a.bins;                                 // [bins] this CTA's totals (peers read it)
+    int32_t *sh = cta_tot + a.bins;                                  // [32] scan scratch
+    const int tile = blockIdx.x * warps + warp;
     const unsigned lt = lanemask_lt();
 
-    const int32_t *base = a.part + (size_t)tile * a.bins;
-    for (int b = lane; b < nb; b += 32)
-        run[b] = base[b] + (b < a.E ? a.out.expert_offsets[b] : a.out.rank_row_offsets[b - a.E]);
-    __syncwarp();
+    EP_STAMP(0);
+    count_tile(a, run, ids, tile, lane);
+    __syncthreads();
+    EP_STAMP(1);
+    // per bin: exclusive prefix over this CTA's warps (in place) and the CTA total
+    for (int b = threadIdx.x; b < a.bins; b += blockDim.x) {
+        int32_t mine = 0;
+        for (int w = 0; w < warps; ++w) {
+            const int32_t v = smem[w * pw + b];
+            smem[w * pw + b] = mine;
+            mine += v;
+        }
+        cta_tot[b] = mine;
+    }
+    if (a.mode == kModeCluster) cg::this_cluster().sync();           // every peer's cta_tot is written
+    else if (a.mode == kModeGlobal) asm volatile("griddepcontrol.wait;" ::: "memory");   // cta_part is complete and visible
+    else __syncthreads();
+    EP_STAMP(2);
+    // per bin: count in earlier CTAs and grand total
+    for (int b = threadIdx.x; b < a.bins; b += blockDim.x) {
+        int32_t before = 0, total = 0;
+        if (a.mode == kModeCluster) {
+            cg::cluster_group cluster = cg::this_cluster();
+#pragma unroll 8
+            for (int c = 0; c < a.n_ctas; ++c) {
+                const int32_t v = cluster.map_shared_rank(cta_tot, c)[b];
+                total += v;
+                if (c < (int)blockIdx.x) before += v;
+            }
+        } else if (a.mode == kModeGlobal) {
+#pragma unroll 16
+            for (int c = 0; c < a.n_ctas; ++c) {
+                const int32_t v = __ldcg(a.cta_part + (size_t)c * a.bins + b);
+                total += v;
+                if (c < (int)blockIdx.x) before += v;
+            }
+        } else {
+            total = cta_tot[b];
+        }
+        pre[b] = before;
+        if (b < a.E) tot_e[b] = total;
+        else if (b < nb) tot_r[b - a.E] = total;
+        if (blockIdx.x == 0) {
+            if (b < a.E) a.out.expert_counts[b] = total;
+            else if (b < nb) a.out.rank_rows[b - a.E] = total;
+            else *a.out.status = total ? EP_STATUS_BAD_INDEX : 0;
+        }
+    }
+    if (a.mode == kModeCluster) cg::this_cluster().sync();           // peers are done with this CTA's shared memory
+    else __syncthreads();
+    EP_STAMP(3);
+    block_exclusive_scan_smem(tot_e, a.E, sh);
+    block_exclusive_scan_smem(tot_r, a.R, sh);
+    if (blockIdx.x == 0) {
+        for (int e = threadIdx.x; e <= a.E; e += blockDim.x) a.out.expert_offsets[e] = tot_e[e];
+        for (int r = threadIdx.x; r <= a.R; r += blockDim.x) a.out.rank_row_offsets[r] = tot_r[r];
+        for (int r = threadIdx.x; r < a.R; r += blockDim.x) a.out.src_row_offsets[r * (a.R + 1) + a.R] = tot_r[r + 1];
+    }
+    for (int b = threadIdx.x; b < nb; b += blockDim.x) {
+        const int32_t base = pre[b] + (b < a.E ? tot_e[b] : tot_r[b - a.E]);
+        for (int w = 0; w < warps; ++w) smem[w * pw + b] += base;
+    }
+    __syncthreads();
+    EP_STAMP(4);
+    if (tile >= a.n_tiles) return;
 
+    // replay the tile in (t,k) order; run[bin] = next free slot of the bin
     const int t0 = tile * a.tile_tokens;
     const int t1 = min(a.T, t0 + a.tile_tokens);
     for (int tb = t0; tb < t1; tb += 32) {
         const int t = tb + lane;
         const bool live = t < t1;
+        const int n_items = stage_group(a, ids, tb, t1, lane);
         // --- receive rows: which of these 32 tokens hit which rank
-        unsigned long long mask = 0ull;
-        if (live)
-            for (int k = 0; k < a.K; ++k) {
-                const int e = __ldg(a.idx + (size_t)t * a.K + k);
-                if (e >= 0 && e < a.E) mask |= 1ull << (e / a.El);
-            }
+        const unsigned long long mask = token_rank_mask(a, ids, lane);
         for (int r = 0; r < a.R; ++r) {
             const unsigned b = __ballot_sync(kFullMask, (mask >> r) & 1ull);
             if (lane == 0) bal[r] = b;
         }
         __syncwarp();
         if (live) {
-            if (t % a.Tr == 0) {                     // first token of a source rank
-                const int s = t / a.Tr;
+            const int s = fdiv(t, a.by_Tr);
+            if (t == s * a.Tr)                       // first token of source rank s
                 for (int r = 0; r < a.R; ++r)
                     a.out.src_row_offsets[r * (a.R + 1) + s] = run[a.E + r] + __popc(bal[r] & lt);
-            }
             unsigned long long seen = 0ull;
             for (int k = 0; k < a.K; ++k) {
-                const int e = __ldg(a.idx + (size_t)t * a.K + k);
+                const int e = ids[lane * a.K + k];
                 int32_t row = -1;
                 if (e >= 0 && e < a.E) {
-                    const int r = e / a.El;
+                    const int r = fdiv(e, a.by_El);
                     row = run[a.E + r] + __popc(bal[r] & lt);
                     if (!((seen >> r) & 1ull)) {
                         a.out.recv_token[row] = t;
@@ -236,12 +346,12 @@ __global__ void layout_assign_kernel(LayoutArgs a)
         for (int r = lane; r < a.R; r += 32) run[a.E + r] += __popc(bal[r]);
         __syncwarp();
         // --- pair slots: the items of these tokens, 32 at a time in (t,k) order
-        const int n_items = (min(t1, tb + 32) - tb) * a.K;
-        const size_t i0 = (size_t)tb * a.K;
+        int32_t *pair_slot = a.out.pair_slot + (size_t)tb * a.K;
+        int32_t *recv_slot = a.out.recv_slot + (size_t)tb * a.K;
         for (int j = 0; j < n_items; j += 32) {
             const int i = j + lane;
             const bool act = i < n_items;
-            const int e = act ? __ldg(a.idx + i0 + i) : -1;
+            const int e = act ? ids[i] : -1;
             const bool valid = act && e >= 0 && e < a.E;
             const unsigned m = __match_any_sync(kFullMask, valid ? e : a.E + lane);
             int32_t first = 0;
@@ -249,23 +359,28 @@ __global__ void layout_assign_kernel(LayoutArgs a)
                 first = run[e];
                 const int32_t p = first + __popc(m & lt);
                 const int32_t row = slot_s[i];
-                a.out.pair_slot[i0 + i] = p;
-                a.out.recv_slot[i0 + i] = row;
-                a.out.pair_token[p] = tb + i / a.K;
+                pair_slot[i] = p;
+                recv_slot[i] = row;
+                a.out.pair_token[p] = tb + fdiv(i, a.by_K);
                 a.out.pair_row[p] = row;
             } else if (act) {
-                a.out.pair_slot[i0 + i] = -1;
-                a.out.recv_slot[i0 + i] = -1;
+                pair_slot[i] = -1;
+                recv_slot[i] = -1;
             }
             __syncwarp();
             if (valid && (m >> lane) <= 1u) run[e] = first + __popc(m);   // highest lane of the group
             __syncwarp();
         }
+        EP_STAMP(5 + (tb - t0) / 32);
     }
 }
 
 }  // namespace
 }  // namespace ep
+
+#ifdef EP_LAYOUT_TIMING
+extern "C" void ep_debug_set_timing_buffer(long long *p) { ep::g_timing_buf = p; }
+#endif
 
 extern "C" size_t ep_layout_workspace_bytes(const ep_shape_t *shape)
 {
@@ -305,25 +420,48 @@ extern "C" int ep_layout(const ep_shape_t *shape, const int32_t *topk_idx, const
     LayoutArgs a;
     a.idx = topk_idx;
     a.out = *out;
-    a.part = static_cast<int32_t *>(workspace);
-    a.totals = a.part + (size_t)plan.n_tiles * plan.bins;
-    a.ticket = reinterpret_cast<unsigned *>(a.totals + plan.bins);
-    a.T = T; a.K = shape->top_k; a.E = E; a.R = R; a.El = E / R; a.Tr = T / R;
-    a.tile_tokens = plan.tile_tokens; a.n_tiles = plan.n_tiles; a.bins = plan.bins;
+    a.cta_part = static_cast<int32_t *>(workspace);
+    a.T = T; a.K = shape->top_k; a.E = E; a.R = R; a.Tr = T / R;
+    a.by_El = make_fastdiv(E / R); a.by_K = make_fastdiv(shape->top_k); a.by_Tr = make_fastdiv(T / R);
+    a.tile_tokens = plan.tile_tokens; a.n_tiles = plan.n_tiles; a.bins = plan.bins; a.n_ctas = plan.n_ctas;
+    a.mode = plan.mode;
+#ifdef EP_LAYOUT_TIMING
+    a.dbg = g_timing_buf;
+#endif
 
     static bool attr_done[64] = {};
     int dev = 0;
     EP_CUDA_TRY(cudaGetDevice(&dev));
     if (dev < 64 && !attr_done[dev]) {
-        EP_CUDA_TRY(cudaFuncSetAttribute(layout_count_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024));
-        EP_CUDA_TRY(cudaFuncSetAttribute(layout_assign_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024));
+        EP_CUDA_TRY(cudaFuncSetAttribute(layout_cta_count_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget));
+        EP_CUDA_TRY(cudaFuncSetAttribute(layout_assign_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget));
         attr_done[dev] = true;
     }
-    const int grid_tiles = ceil_div(plan.n_tiles, plan.warps);
-    layout_count_kernel<<<grid_tiles, plan.warps * 32, plan.smem_count, stream>>>(a);
-    layout_scan_kernel<<<ceil_div(plan.bins, kScanWarps), kScanWarps * 32, 0, stream>>>(a);
-    layout_assign_kernel<<<grid_tiles, plan.warps * 32, plan.smem_assign, stream>>>(a);
-    EP_LAUNCH_CHECK(3);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(plan.n_ctas);
+    cfg.blockDim = dim3(plan.warps * 32);
+    cfg.dynamicSmemBytes = plan.smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr;
+    int launched = 1;
+    if (plan.mode == kModeCluster) {
+        attr.id = cudaLaunchAttributeClusterDimension;      // the whole grid is one cluster
+        attr.val.clusterDim.x = plan.n_ctas;
+        attr.val.clusterDim.y = 1;
+        attr.val.clusterDim.z = 1;
+        cfg.attrs = &attr;
+        cfg.numAttrs = 1;
+    } else if (plan.mode == kModeGlobal) {
+        layout_cta_count_kernel<<<plan.n_ctas, plan.warps * 32, plan.smem, stream>>>(a);
+        // the main kernel may start while the first still runs; it waits on the device before it reads cta_part
+        attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr.val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = &attr;
+        cfg.numAttrs = 1;
+        launched = 2;
+    }
+    EP_CUDA_TRY(cudaLaunchKernelEx(&cfg, layout_assign_kernel, a));
+    EP_LAUNCH_CHECK(launched);
     return EP_OK;
 }
 

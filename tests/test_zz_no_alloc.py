@@ -36,8 +36,10 @@ def _same(a: ep.Layout, b: ep.Layout):
 def test_static_scratch_layout_matches_ep_layout_on_two_calls_in_a_row():
     assert ep.ep_layout_static_scratch_bytes() == 1 << 20
     # two workloads of different shape and routing, so stale scratch would show
-    first, second = inputs.CONFIGS["C4"], inputs.CONFIGS["C3"]
-    for cfg in (first, second, first):
+    # (the 40000-token batch is past the single-cluster size, so its layout really uses the scratch)
+    big = inputs.custom_config(40000, 8, 16, 2, 8, config_id=78)
+    big2 = inputs.custom_config(65536, 8, 64, 4, 8, routing="zipf", config_id=79)
+    for cfg in (big, inputs.CONFIGS["C4"], big2, big, inputs.CONFIGS["C3"]):
         idx = torch.from_numpy(inputs.make_topk_idx(cfg)).cuda()
         want = ep.alloc_layout(cfg.T, cfg.K, cfg.E, cfg.R, fill=-3)
         ep.ep_layout(idx, cfg.E, cfg.R, out=want)
