@@ -31,7 +31,63 @@ NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes per launch of the dominant kernel from the committed ncu capture
 # (profiles/): filled in per workload once measured, else null.
-NCU_TRAFFIC_BYTES = {}
+NCU_TRAFFIC_BYTES = {("C4", "combine_rows_kernel"): 1038.7e6, ("C4", "dispatch_rows_kernel"): 681.3e6}
+L2_BYTES = 126e6
+
+
+def LAUNCHES_PER_STEP(ep, step):
+    """Kernels one direct (non-graph) step launches, counted by the library."""
+    n0 = ep.ep_launch_count()
+    step()
+    torch.cuda.synchronize()
+    return ep.ep_launch_count() - n0
+
+
+def host_staged_arms(ep, cfg, x, lay, recv_host, dev, iters=10):
+    """Receive buffer in mapped pinned host memory: (i) the dispatch kernel stores straight
+    into it; (ii) dispatch packs into device staging and the copy engine moves each rank's
+    partition; plus the host-link probe both are measured against."""
+    E, R = cfg.E, cfg.R
+    n_recv = int(lay.rank_row_offsets[-1])
+    row = 2 * cfg.H
+    staging = torch.empty(recv_host.shape[0], cfg.H, dtype=torch.bfloat16, device=dev)
+    probe_src = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    probe_dst = torch.empty(256 << 20, dtype=torch.uint8).pin_memory()
+    d2h = ep.ep_probe_bandwidth(ep.PROBE_MEMCPY, probe_dst, probe_src, 256 << 20, iters=10)
+    h2d = ep.ep_probe_bandwidth(ep.PROBE_MEMCPY, probe_src, probe_dst, 256 << 20, iters=10)
+
+    def timed(fn):
+        best = 1e30
+        for _ in range(iters + 1):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            fn()
+            b.record()
+            torch.cuda.synchronize()
+            best = min(best, a.elapsed_time(b))
+        return best
+
+    def arm_kernel():
+        ep.ep_dispatch(x, lay.recv_slot, recv_host, E, R)
+
+    offs_pinned = torch.zeros(R + 1, dtype=torch.int32).pin_memory()
+
+    def arm_copy_known():           # the offsets first travel to the host: one small copy and a stream sync, timed
+        offs_pinned.copy_(lay.rank_row_offsets, non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+        ep.ep_dispatch_copy_engine(x, lay.recv_slot, staging, recv_host, E, R, rank_row_offsets_host=offs_pinned)
+
+    def arm_copy_blind():           # no count reaches the host: one copy of the worst-case T*min(K,R) rows
+        ep.ep_dispatch_copy_engine(x, lay.recv_slot, staging, recv_host, E, R, rank_row_offsets_host=None)
+
+    res = {"host_link_d2h_GB/s": d2h, "host_link_h2d_GB/s": h2d, "rows": n_recv, "bytes_over_link": n_recv * row}
+    for name, fn, nbytes in [("kernel_store", arm_kernel, n_recv * row),
+                             ("copy_engine_per_rank", arm_copy_known, n_recv * row),
+                             ("copy_engine_worst_case", arm_copy_blind, recv_host.shape[0] * row)]:
+        ms = timed(fn)
+        res[name] = {"us": ms * 1e3, "GB/s": nbytes / (ms * 1e-3) / 1e9, "useful_GB/s": n_recv * row / (ms * 1e-3) / 1e9,
+                     "frac_of_d2h_probe": n_recv * row / (ms * 1e-3) / 1e9 / d2h, "tokens/s": cfg.T / (ms * 1e-3)}
+    return res
 
 
 def workload_text(cfg):
@@ -119,36 +175,6 @@ class ClockSampler:
                 "reasons": sorted(self.reasons), "samples": len(self.samples)}
 
 
-def dist_setup(n_gpus):
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
-    if world > 1:
-        import torch.distributed as dist
-        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-        torch.cuda.set_device(local)
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    else:
-        torch.cuda.set_device(0)
-    return rank, world, local
-
-
-def barrier(world):
-    if world > 1:
-        import torch.distributed as dist
-        dist.barrier()
-    torch.cuda.synchronize()
-
-
-def max_over_ranks(value, world):
-    if world == 1:
-        return value
-    import torch.distributed as dist
-    t = torch.tensor([value], dtype=torch.float64, device="cuda")
-    dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    return float(t.item())
-
-
 def cpu_oracle_step(oracle, idx, w, x, out):
     lay = oracle.layout(idx, CPU_CFG.E, CPU_CFG.R)
     oracle.dispatch(x, lay.recv_slot, lay.n_recv)
@@ -225,6 +251,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=20)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="small workloads: time direct launches, not graph replays")
     ap.add_argument("--seed", type=int, default=0)
     args = ap.parse_args()
     if args.warmup < 3:
@@ -238,10 +265,12 @@ def main():
 
     import __graft_entry__ as entry
     from paper_2609_40093_b200 import ep
-    rank, world, local = dist_setup(args.gpus)
+    from paper_2609_40093_b200.replicas import Replicas
+    rep = Replicas()
+    rank, world = rep.rank, rep.world
     if rank == 0:
         entry.build()
-    barrier(world)
+    rep.barrier()
     dev = torch.device("cuda", torch.cuda.current_device())
     rcfg = inputs.shard_config(cfg, rank)            # replica `rank`: same shapes, its own seed stream
     T, K, H, E, R = cfg.T, cfg.K, cfg.H, cfg.E, cfg.R
@@ -282,24 +311,72 @@ def main():
     assert ep.ep_status(lay.status) == 0
     n_recv, n_pairs = int(lay.rank_row_offsets[-1]), int(lay.expert_offsets[-1])
     alg = algorithmic_bytes(cfg, n_recv, n_pairs)
+    step_bytes = alg["dispatch"] + alg["combine"]
+    small = step_bytes < 4 * L2_BYTES and not cfg.host_staged       # the step's data could (partly) stay in L2
 
-    # ---- timed region: K steps, device-timed, per-kernel events on the launching stream
-    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
-    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     launches0 = ep.ep_launch_count()
-    barrier(world)
-    with ClockSampler(torch.cuda.current_device()) as clocks:
-        start.record()
-        for i in range(args.steps):
-            step(evs[i])
-        stop.record()
+    if not small:
+        # ---- timed region: K steps back to back, device-timed, per-kernel events on the launching stream
+        evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
+        start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        rep.barrier()
+        with ClockSampler(torch.cuda.current_device()) as clocks:
+            start.record()
+            for i in range(args.steps):
+                step(evs[i])
+            stop.record()
+            torch.cuda.synchronize()
+        rep.barrier()
+        launches = ep.ep_launch_count() - launches0
+        total_ms = rep.max_over_ranks(start.elapsed_time(stop))
+        per = np.array([[e[j].elapsed_time(e[j + 1]) for j in range(3)] for e in evs])  # ms: layout, dispatch, combine
+        l2_note = "working set per step exceeds L2 several times over (no flush needed)"
+        launch_note = "direct launches"
+    else:
+        # ---- small workloads: L2 is flushed (256 MB written) before every step; each step is timed by its own
+        # event pair and the step itself is a CUDA-graph replay, so host launch cost is not what is measured
+        flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+        graph = None
+        if not args.no_graph:
+            side = torch.cuda.Stream()
+            with torch.cuda.stream(side):
+                step()
+            torch.cuda.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph):
+                step()
+        s_ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+        e_ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
+        rep.barrier()
+        with ClockSampler(torch.cuda.current_device()) as clocks:
+            for i in range(args.steps):
+                flush.fill_(i & 0xff)
+                s_ev[i].record()
+                graph.replay() if graph is not None else step()
+                e_ev[i].record()
+            torch.cuda.synchronize()
+        rep.barrier()
+        launches = ep.ep_launch_count() - launches0
+        if graph is not None:                   # replays launch the captured kernels without passing through the library
+            launches = args.steps * LAUNCHES_PER_STEP(ep, step)
+        total_ms = rep.max_over_ranks(sum(s.elapsed_time(e) for s, e in zip(s_ev, e_ev)))
+        # per-kernel figures from a separate pass of direct launches, each step after a flush
+        evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(min(args.steps, 50))]
+        for e in evs:
+            flush.fill_(1)
+            step(e)
         torch.cuda.synchronize()
-    barrier(world)
-    launches = ep.ep_launch_count() - launches0
-    total_ms = max_over_ranks(start.elapsed_time(stop), world)
-    per = np.array([[e[j].elapsed_time(e[j + 1]) for j in range(3)] for e in evs])      # ms: layout, dispatch, combine
+        per = np.array([[e[j].elapsed_time(e[j + 1]) for j in range(3)] for e in evs])
+        l2_note = "step data would fit L2: 256 MB flush write before every timed step, each step timed by its own event pair"
+        launch_note = "CUDA graph replay of one step" if graph is not None else "direct launches"
+        del flush
     lay_ms, dis_ms, com_ms = [float(v) for v in per.mean(axis=0)]
     value = world * T * args.steps / (total_ms * 1e-3)
+
+    # ---- host-staged variant: the two arms of the receive path and the host-link probe
+    host = None
+    if cfg.host_staged:
+        host = host_staged_arms(ep, cfg, x, lay, recv, dev)
 
     # ---- end to end: one C-ABI call per step, host buffers in, host buffer out
     arena = torch.empty(ep.ep_host_step_arena_bytes(T, K, H, E, R), dtype=torch.uint8, device=dev)
@@ -308,14 +385,14 @@ def main():
     n_e2e = max(1, args.e2e_steps)
     for _ in range(3 if args.e2e_steps > 0 else 0):
         ep.ep_host_step(x_h, idx_h, w_h, y_h, arena, E, R, status_host=st_h)
-    barrier(world)
+    rep.barrier()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for _ in range(args.e2e_steps):
         ep.ep_host_step(x_h, idx_h, w_h, y_h, arena, E, R, status_host=st_h)
     e1.record()
     torch.cuda.synchronize()
-    e2e_ms = max_over_ranks(e0.elapsed_time(e1), world)
+    e2e_ms = rep.max_over_ranks(e0.elapsed_time(e1))
     assert int(st_h[0]) == 0
     e2e_value = world * T * args.e2e_steps / (e2e_ms * 1e-3) if args.e2e_steps > 0 else None
     h2d = x_h.numel() * 2 + idx_h.numel() * 4 + w_h.numel() * 4
@@ -323,9 +400,7 @@ def main():
     del arena
 
     if rank != 0:
-        if world > 1:
-            import torch.distributed as dist
-            dist.destroy_process_group()
+        rep.close()
         return
     peak, peak_kind = measured_peak()
     com_gbs = alg["combine"] / (com_ms * 1e-3) / 1e9
@@ -341,8 +416,7 @@ def main():
         "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": workload_text(cfg), "parallelism": f"{world} independent replica(s)",
-                   "l2": "working set per step exceeds L2 (no flush needed)" if alg["combine"] > 2 * 126e6
-                   else "working set fits L2: warm-L2 latency figures", "n_recv": n_recv, "n_pairs": n_pairs},
+                   "l2": l2_note, "launch": launch_note, "n_recv": n_recv, "n_pairs": n_pairs},
         "ops": {
             "layout": {"us": lay_ms * 1e3},
             "dispatch": {"us": dis_ms * 1e3, "GB/s": dis_gbs, "tokens/s": T / (dis_ms * 1e-3), "bytes": alg["dispatch"]},
@@ -358,6 +432,13 @@ def main():
         "context": "paper reports 2.00x (dispatch) / 1.53x (combine) over NCCL for its dense all-gather/"
                    "reduce-scatter on RTX 4090/5090 PCIe boxes; no number for the routing-aware path",
     }
+    if host is not None:
+        line["host_staged"] = host
+        link = host["host_link_d2h_GB/s"]
+        line["roofline_dispatch"] = {"bound": "host-link", "kernel": "dispatch_rows_kernel (stores to mapped pinned memory)",
+                                     "achieved": host["kernel_store"]["GB/s"], "peak": link,
+                                     "peak_kind": "cudaMemcpyAsync D2H probe, 256 MB pinned, same run", "unit": "GB/s",
+                                     "frac": host["kernel_store"]["GB/s"] / link, "traffic": None}
     if not args.no_cpu_baseline:
         out_h = out.view(torch.int16).cpu().numpy().view(np.uint16)
         v, n, el = time_oracle(cfg, d["topk_idx"], d["topk_weights"], d["x"], out_h, min_seconds=10.0, max_steps=20)
@@ -365,9 +446,7 @@ def main():
                                 "sample": f"{n} whole step(s) of the same {cfg.name} batch in {el:.1f} s, one thread",
                                 "host_cores_available": os.cpu_count()}
     print(json.dumps(line))
-    if world > 1:
-        import torch.distributed as dist
-        dist.destroy_process_group()
+    rep.close()
 
 
 if __name__ == "__main__":
