@@ -1,16 +1,48 @@
 // ep_dispatch / ep_group: row movers. One bf16 row is H/8 16-byte vectors; a group of
-// G threads (G = 32, 64 or 128, chosen from the row length) owns one source row,
-// loads up to kVecPerThread vectors per thread into registers once, and stores
-// them to every destination row. Each warp finds its row's distinct destinations
-// by itself (K <= 32 slots, one per lane, duplicates dropped with a warp match),
-// so there is no shared memory and no block-wide barrier.
+// G threads (a multiple of 32, chosen from the row length) owns one source row,
+// loads U vectors per thread into registers once, and stores them to every
+// destination row. Each warp finds its row's distinct destinations by itself
+// (K <= 32 slots, one per lane, duplicates dropped with a warp match), so there
+// is no shared memory and no block-wide barrier.
+#include <cstdio>
+#include <cstdlib>
+
 #include "ep_common.cuh"
 
 namespace ep {
 namespace {
 
-constexpr int kBlock = 128;
-constexpr int kVecPerThread = 8;
+constexpr int kMinBlock = 128;
+
+// Thread group per row and vectors per thread: G*U covers the row when it can
+// (long rows: many threads with one or two vectors each; short rows: one warp).
+struct RowPlan {
+    int G, U, block, rows_per_block;
+};
+
+RowPlan plan_rows(int vec_per_row, const char *tune_env)
+{
+    RowPlan p;
+    // two vectors per thread, up to 512 threads per row (measured: the row movers are HBM-bound for any
+    // G at H=7168; at H=2048, T=4096 more threads per row shorten the kernel by ~8 %)
+    int G = ceil_div(ceil_div(vec_per_row, 2), 32) * 32, U = 2;
+    if (G > 512) G = 512;
+    if (vec_per_row <= 32) U = 1;
+#ifdef EP_TUNING
+    if (const char *e = getenv(tune_env)) {      // "G,U" override, tuning builds only
+        int g = 0, u = 0;
+        if (sscanf(e, "%d,%d", &g, &u) == 2 && g >= 32 && g % 32 == 0 && (u == 1 || u == 2 || u == 4 || u == 8) &&
+            g <= (u == 8 ? 256 : (u == 4 ? 512 : 1024))) { G = g; U = u; }
+    }
+#else
+    (void)tune_env;
+#endif
+    p.G = G;
+    p.U = U;
+    p.rows_per_block = G >= kMinBlock ? 1 : kMinBlock / G;
+    p.block = G * p.rows_per_block;
+    return p;
+}
 
 __device__ __forceinline__ void flag_status(int32_t *status, int bits)
 {
@@ -18,15 +50,15 @@ __device__ __forceinline__ void flag_status(int32_t *status, int bits)
 }
 
 // recv[recv_slot[t][k]] = x[t] for the distinct slots of token t.
-template <int G>
-__global__ void __launch_bounds__(kBlock)
+template <int U>
+__global__ void __launch_bounds__(U >= 8 ? 256 : (U == 4 ? 512 : 1024))
 dispatch_rows_kernel(const uint4 *__restrict__ x, const int32_t *__restrict__ recv_slot, uint4 *recv,
-                     int T, int K, int vec_per_row, long long capacity_rows, int32_t *status)
+                     int T, int K, int vec_per_row, int G, long long capacity_rows, int32_t *status)
 {
     const int lane = threadIdx.x & 31;
     const int g = threadIdx.x % G;                       // position inside the row group
-    const int t = blockIdx.x * (kBlock / G) + threadIdx.x / G;
-    if (t >= T) return;                                   // whole warps leave together (G >= 32)
+    const int t = blockIdx.x * (blockDim.x / G) + threadIdx.x / G;
+    if (t >= T) return;                                   // whole warps leave together (G % 32 == 0)
 
     int32_t slot = lane < K ? __ldg(recv_slot + (size_t)t * K + lane) : -1;
     if (slot >= capacity_rows) {
@@ -38,11 +70,11 @@ dispatch_rows_kernel(const uint4 *__restrict__ x, const int32_t *__restrict__ re
     unsigned todo = __ballot_sync(kFullMask, slot >= 0 && (same & lanemask_lt()) == 0);
 
     const uint4 *src = x + (size_t)t * vec_per_row;
-    for (int base = 0; base < vec_per_row; base += G * kVecPerThread) {  // trip count uniform over the warp
+    for (int base = 0; base < vec_per_row; base += G * U) {  // trip count uniform over the warp
         const int v0 = base + g;
-        uint4 buf[kVecPerThread];
+        uint4 buf[U];
 #pragma unroll
-        for (int u = 0; u < kVecPerThread; ++u) {
+        for (int u = 0; u < U; ++u) {
             const int v = v0 + u * G;
             if (v < vec_per_row) buf[u] = ld_stream(src + v);
         }
@@ -50,7 +82,7 @@ dispatch_rows_kernel(const uint4 *__restrict__ x, const int32_t *__restrict__ re
             const int32_t row = __shfl_sync(kFullMask, slot, __ffs(m) - 1);
             uint4 *dst = recv + (size_t)row * vec_per_row;
 #pragma unroll
-            for (int u = 0; u < kVecPerThread; ++u) {
+            for (int u = 0; u < U; ++u) {
                 const int v = v0 + u * G;
                 if (v < vec_per_row) st_stream(dst + v, buf[u]);
             }
@@ -59,14 +91,14 @@ dispatch_rows_kernel(const uint4 *__restrict__ x, const int32_t *__restrict__ re
 }
 
 // grouped[p] = recv[pair_row[p]] for p < P = *n_pairs.
-template <int G>
-__global__ void __launch_bounds__(kBlock)
+template <int U>
+__global__ void __launch_bounds__(U >= 8 ? 256 : (U == 4 ? 512 : 1024))
 group_rows_kernel(const uint4 *__restrict__ recv, long long recv_rows, const int32_t *__restrict__ pair_row,
                   const int32_t *__restrict__ n_pairs, uint4 *grouped, long long capacity_rows,
-                  int vec_per_row, int32_t *status)
+                  int vec_per_row, int G, int32_t *status)
 {
     const int g = threadIdx.x % G;
-    const long long p = (long long)blockIdx.x * (kBlock / G) + threadIdx.x / G;
+    const long long p = (long long)blockIdx.x * (blockDim.x / G) + threadIdx.x / G;
     if (p >= __ldg(n_pairs)) return;
     if (p >= capacity_rows) {
         if (g == 0) flag_status(status, EP_STATUS_CAPACITY);
@@ -79,26 +111,19 @@ group_rows_kernel(const uint4 *__restrict__ recv, long long recv_rows, const int
     }
     const uint4 *src = recv + (size_t)row * vec_per_row;
     uint4 *dst = grouped + (size_t)p * vec_per_row;
-    for (int v0 = g; v0 < vec_per_row; v0 += G * kVecPerThread) {
-        uint4 buf[kVecPerThread];
+    for (int v0 = g; v0 < vec_per_row; v0 += G * U) {
+        uint4 buf[U];
 #pragma unroll
-        for (int u = 0; u < kVecPerThread; ++u) {
+        for (int u = 0; u < U; ++u) {
             const int v = v0 + u * G;
             if (v < vec_per_row) buf[u] = ld_stream(src + v);
         }
 #pragma unroll
-        for (int u = 0; u < kVecPerThread; ++u) {
+        for (int u = 0; u < U; ++u) {
             const int v = v0 + u * G;
             if (v < vec_per_row) st_stream(dst + v, buf[u]);
         }
     }
-}
-
-int pick_group(int vec_per_row)
-{
-    if (vec_per_row <= 32 * kVecPerThread) return 32;
-    if (vec_per_row <= 64 * kVecPerThread) return 64;
-    return 128;
 }
 
 }  // namespace
@@ -109,15 +134,13 @@ int launch_dispatch(const ep_shape_t &s, const void *x, const int32_t *recv_slot
     const int T = s.num_tokens, K = s.top_k, vpr = s.hidden / 8;
     const uint4 *xs = static_cast<const uint4 *>(x);
     uint4 *rd = static_cast<uint4 *>(recv);
-    switch (pick_group(vpr)) {
-    case 32:
-        dispatch_rows_kernel<32><<<ceil_div(T, kBlock / 32), kBlock, 0, stream>>>(xs, recv_slot, rd, T, K, vpr, capacity_rows, status);
-        break;
-    case 64:
-        dispatch_rows_kernel<64><<<ceil_div(T, kBlock / 64), kBlock, 0, stream>>>(xs, recv_slot, rd, T, K, vpr, capacity_rows, status);
-        break;
-    default:
-        dispatch_rows_kernel<128><<<T, kBlock, 0, stream>>>(xs, recv_slot, rd, T, K, vpr, capacity_rows, status);
+    const RowPlan p = plan_rows(vpr, "EP_TUNE_DISPATCH");
+    const int grid = ceil_div(T, p.rows_per_block);
+    switch (p.U) {
+    case 1: dispatch_rows_kernel<1><<<grid, p.block, 0, stream>>>(xs, recv_slot, rd, T, K, vpr, p.G, capacity_rows, status); break;
+    case 2: dispatch_rows_kernel<2><<<grid, p.block, 0, stream>>>(xs, recv_slot, rd, T, K, vpr, p.G, capacity_rows, status); break;
+    case 4: dispatch_rows_kernel<4><<<grid, p.block, 0, stream>>>(xs, recv_slot, rd, T, K, vpr, p.G, capacity_rows, status); break;
+    default: dispatch_rows_kernel<8><<<grid, p.block, 0, stream>>>(xs, recv_slot, rd, T, K, vpr, p.G, capacity_rows, status);
     }
     EP_LAUNCH_CHECK(1);
     return EP_OK;
@@ -131,15 +154,13 @@ int launch_group(const ep_shape_t &s, const void *recv, int64_t recv_rows, const
     const int vpr = s.hidden / 8;
     const uint4 *rs = static_cast<const uint4 *>(recv);
     uint4 *gd = static_cast<uint4 *>(grouped);
-    switch (pick_group(vpr)) {
-    case 32:
-        group_rows_kernel<32><<<(unsigned)((max_pairs + 3) / 4), kBlock, 0, stream>>>(rs, recv_rows, pair_row, n_pairs, gd, capacity_rows, vpr, status);
-        break;
-    case 64:
-        group_rows_kernel<64><<<(unsigned)((max_pairs + 1) / 2), kBlock, 0, stream>>>(rs, recv_rows, pair_row, n_pairs, gd, capacity_rows, vpr, status);
-        break;
-    default:
-        group_rows_kernel<128><<<(unsigned)max_pairs, kBlock, 0, stream>>>(rs, recv_rows, pair_row, n_pairs, gd, capacity_rows, vpr, status);
+    const RowPlan p = plan_rows(vpr, "EP_TUNE_GROUP");
+    const unsigned grid = (unsigned)((max_pairs + p.rows_per_block - 1) / p.rows_per_block);
+    switch (p.U) {
+    case 1: group_rows_kernel<1><<<grid, p.block, 0, stream>>>(rs, recv_rows, pair_row, n_pairs, gd, capacity_rows, vpr, p.G, status); break;
+    case 2: group_rows_kernel<2><<<grid, p.block, 0, stream>>>(rs, recv_rows, pair_row, n_pairs, gd, capacity_rows, vpr, p.G, status); break;
+    case 4: group_rows_kernel<4><<<grid, p.block, 0, stream>>>(rs, recv_rows, pair_row, n_pairs, gd, capacity_rows, vpr, p.G, status); break;
+    default: group_rows_kernel<8><<<grid, p.block, 0, stream>>>(rs, recv_rows, pair_row, n_pairs, gd, capacity_rows, vpr, p.G, status);
     }
     EP_LAUNCH_CHECK(1);
     return EP_OK;
