@@ -119,3 +119,57 @@ def combine_f64(out_bits: np.ndarray, slot: np.ndarray, w: np.ndarray) -> np.nda
     if rc != 0:
         raise ValueError("oracle combine: slot beyond out rows")
     return y
+
+
+def group(recv_bits: np.ndarray, pair_row: np.ndarray) -> np.ndarray:
+    recv = np.ascontiguousarray(recv_bits, dtype=np.uint16)
+    pr = np.ascontiguousarray(pair_row, dtype=np.int32)
+    H = recv.shape[1]
+    grouped = np.zeros((pr.shape[0], H), dtype=np.uint16)
+    rc = _load().ep_oracle_group(ctypes.c_int64(pr.shape[0]), H, _p(recv), ctypes.c_int64(recv.shape[0]), _p(pr),
+                                 _p(grouped))
+    if rc != 0:
+        raise ValueError("oracle group: pair_row outside the receive buffer")
+    return grouped
+
+
+def combine_partial(out_bits, pair_slot, recv_slot, w, recv_rows: int, fill: int = 0):
+    """Two-stage combine with per-rank partial outputs; returns (partial [recv_rows,H], y [T,H])."""
+    out = np.ascontiguousarray(out_bits, dtype=np.uint16)
+    ps = np.ascontiguousarray(pair_slot, dtype=np.int32)
+    rs = np.ascontiguousarray(recv_slot, dtype=np.int32)
+    wt = np.ascontiguousarray(w, dtype=np.float32)
+    T, K = ps.shape
+    H = out.shape[1]
+    partial = np.full((recv_rows, H), fill, dtype=np.uint16)
+    y = np.zeros((T, H), dtype=np.uint16)
+    rc = _load().ep_oracle_combine_partial(T, K, H, _p(out), ctypes.c_int64(out.shape[0]), _p(ps), _p(rs), _p(wt),
+                                           _p(partial), ctypes.c_int64(recv_rows), _p(y))
+    if rc != 0:
+        raise ValueError("oracle combine_partial: slot outside its buffer")
+    return partial, y
+
+
+def dense_allgather(x_bits: np.ndarray, R: int) -> np.ndarray:
+    x = np.ascontiguousarray(x_bits, dtype=np.uint16)
+    T, H = x.shape
+    g = np.zeros((R * T, H), dtype=np.uint16)
+    _load().ep_oracle_dense_allgather(T, H, R, _p(x), _p(g))
+    return g
+
+
+def dense_reduce_scatter(topk_idx, out_bits, pair_slot, w, E: int, R: int):
+    """Dense per-rank buffers ordered by source token and their R-way sum; returns (dense [R*T,H], y [T,H])."""
+    idx = np.ascontiguousarray(topk_idx, dtype=np.int32)
+    out = np.ascontiguousarray(out_bits, dtype=np.uint16)
+    ps = np.ascontiguousarray(pair_slot, dtype=np.int32)
+    wt = np.ascontiguousarray(w, dtype=np.float32)
+    T, K = idx.shape
+    H = out.shape[1]
+    dense = np.zeros((R * T, H), dtype=np.uint16)
+    y = np.zeros((T, H), dtype=np.uint16)
+    rc = _load().ep_oracle_dense_reduce_scatter(T, K, H, E, R, _p(idx), _p(out), ctypes.c_int64(out.shape[0]), _p(ps),
+                                                _p(wt), _p(dense), _p(y))
+    if rc != 0:
+        raise ValueError("oracle dense_reduce_scatter: bad shape or slot")
+    return dense, y

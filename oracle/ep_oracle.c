@@ -213,3 +213,110 @@ int ep_oracle_combine_f64(int T, int K, int H, const uint16_t *out, int64_t out_
         }
     return 0;
 }
+
+/* ------------------------------------------------------------------------
+ * Variants around the path (Section 2.1, "Communication patterns of dispatch
+ * and combine"; Section 4.3).
+ * ------------------------------------------------------------------------ */
+
+/*
+ * Local grouping by expert (Section 4.3: each device groups the tokens it
+ * received by the experts it owns): grouped[p] = recv[pair_row[p]].
+ */
+int ep_oracle_group(int64_t n_pairs, int H, const uint16_t *recv, int64_t recv_rows,
+                    const int32_t *pair_row, uint16_t *grouped)
+{
+    for (int64_t p = 0; p < n_pairs; ++p) {
+        if (pair_row[p] < 0 || pair_row[p] >= recv_rows) return -1;
+        memcpy(grouped + (size_t)p * H, recv + (size_t)pair_row[p] * H, (size_t)H * sizeof(uint16_t));
+    }
+    return 0;
+}
+
+/*
+ * Combine with partial outputs (Section 2.1: an All-to-Allv "transfers only the
+ * tokens and partial outputs required"): every destination rank first sums, per
+ * token it received, the weighted outputs of its own experts, and sends that one
+ * row back; the owner adds the rows of the ranks the token reached.
+ *   stage 1, for each receive row rho = recv_slot[t][k] (one per (t, rank)):
+ *     partial[rho] = bf16( fp32 fma chain over the k' (ascending) of token t
+ *                          with recv_slot[t][k'] == rho of w[t][k']*out[pair_slot[t][k']] )
+ *   stage 2, for each token: y[t] = bf16( fp32 sum, from +0, of partial[rho] over
+ *     the token's distinct receive rows in the order of their first k ).
+ * partial has recv_rows rows; rows no token names are left untouched.
+ */
+int ep_oracle_combine_partial(int T, int K, int H, const uint16_t *out, int64_t out_rows,
+                              const int32_t *pair_slot, const int32_t *recv_slot, const float *w,
+                              uint16_t *partial, int64_t recv_rows, uint16_t *y)
+{
+    for (int t = 0; t < T; ++t)
+        for (int h = 0; h < H; ++h) {
+            float total = 0.0f;
+            for (int k = 0; k < K; ++k) {
+                const int32_t rho = recv_slot[(size_t)t * K + k];
+                if (rho < 0) continue;
+                if (rho >= recv_rows) return -1;
+                int first = 1;
+                for (int k2 = 0; k2 < k; ++k2)
+                    if (recv_slot[(size_t)t * K + k2] == rho) first = 0;
+                if (!first) continue;
+                float acc = 0.0f;                                   /* stage 1 on the expert's rank */
+                for (int k2 = k; k2 < K; ++k2) {
+                    if (recv_slot[(size_t)t * K + k2] != rho) continue;
+                    const int32_t p = pair_slot[(size_t)t * K + k2];
+                    if (p < 0 || p >= out_rows) return -1;
+                    acc = fmaf(w[(size_t)t * K + k2], bf16_to_f32(out[(size_t)p * H + h]), acc);
+                }
+                const uint16_t sent = f32_to_bf16_rne(acc);          /* what travels back */
+                partial[(size_t)rho * H + h] = sent;
+                total = total + bf16_to_f32(sent);                   /* stage 2 on the owner */
+            }
+            y[(size_t)t * H + h] = f32_to_bf16_rne(total);
+        }
+    return 0;
+}
+
+/*
+ * Dense formulation (Section 2.1: All-Gather and Reduce-Scatter; Figure 3).
+ * Dispatch: every rank gathers the tokens of all ranks: gathered[r][t] = x[t],
+ * R*T rows whatever the routing.
+ */
+int ep_oracle_dense_allgather(int T, int H, int R, const uint16_t *x, uint16_t *gathered)
+{
+    for (int r = 0; r < R; ++r)
+        memcpy(gathered + (size_t)r * T * H, x, (size_t)T * H * sizeof(uint16_t));
+    return 0;
+}
+
+/*
+ * Dense combine: rank r places its partial outputs in a dense buffer ordered by
+ * source token, dense[r][t] = bf16( fma chain over the k (ascending) whose expert
+ * lives on r ), +0 where the token has no expert on r; the reduce-scatter returns
+ * y[t] = bf16( fp32 sum from +0 over r = 0..R-1 of dense[r][t] ) to the owner.
+ */
+int ep_oracle_dense_reduce_scatter(int T, int K, int H, int E, int R, const int32_t *topk_idx,
+                                   const uint16_t *out, int64_t out_rows, const int32_t *pair_slot,
+                                   const float *w, uint16_t *dense, uint16_t *y)
+{
+    if (E % R != 0) return -1;
+    const int El = E / R;
+    for (int t = 0; t < T; ++t)
+        for (int h = 0; h < H; ++h) {
+            float total = 0.0f;
+            for (int r = 0; r < R; ++r) {
+                float acc = 0.0f;
+                for (int k = 0; k < K; ++k) {
+                    const int e = topk_idx[(size_t)t * K + k];
+                    if (e < 0 || e >= E || e / El != r) continue;
+                    const int32_t p = pair_slot[(size_t)t * K + k];
+                    if (p < 0 || p >= out_rows) return -1;
+                    acc = fmaf(w[(size_t)t * K + k], bf16_to_f32(out[(size_t)p * H + h]), acc);
+                }
+                const uint16_t placed = f32_to_bf16_rne(acc);
+                dense[((size_t)r * T + t) * H + h] = placed;
+                total = total + bf16_to_f32(placed);
+            }
+            y[(size_t)t * H + h] = f32_to_bf16_rne(total);
+        }
+    return 0;
+}
