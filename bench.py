@@ -43,6 +43,50 @@ def LAUNCHES_PER_STEP(ep, step):
     return ep.ep_launch_count() - n0
 
 
+def time_variants(ep, cfg, idx, w, x, out, lay, n_recv, n_pairs, dev, iters=20):
+    """Median device time of the variants around the path on the same batch: local grouping,
+    expanded dispatch, combine with per-rank partial outputs, dense all-gather / reduce-scatter."""
+    T, K, H, E, R = cfg.T, cfg.K, cfg.H, cfg.E, cfg.R
+    row = 2 * H
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    recv = torch.empty(max(1, n_recv), H, dtype=torch.bfloat16, device=dev)
+    ep.ep_dispatch(x, lay.recv_slot, recv, E, R)
+    y = torch.empty(T, H, dtype=torch.bfloat16, device=dev)
+    res = {"rows": {"routed_receive": n_recv, "pairs": n_pairs, "dense": R * T}}
+
+    def timed(fn, nbytes):
+        ts = []
+        for _ in range(iters + 2):
+            flush.fill_(1)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            fn()
+            b.record()
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b))
+        ms = float(np.median(ts[2:]))
+        return {"us": ms * 1e3, "GB/s": nbytes / (ms * 1e-3) / 1e9, "bytes": nbytes}
+
+    grouped = torch.empty(max(1, n_pairs), H, dtype=torch.bfloat16, device=dev)
+    res["group (recv -> pair rows)"] = timed(lambda: ep.ep_group(recv, lay, grouped, E, R), 2 * row * n_pairs + 4 * n_pairs)
+    res["expanded dispatch (x -> pair rows)"] = timed(lambda: ep.ep_dispatch(x, lay.pair_slot, grouped, E, R),
+                                                      row * T + row * n_pairs + 4 * T * K)
+    del grouped
+    partial = torch.empty(max(1, n_recv), H, dtype=torch.bfloat16, device=dev)
+    res["combine with partial outputs (2 kernels)"] = timed(
+        lambda: ep.ep_combine_partial(out, lay, w, partial, y, E, R),
+        row * n_pairs + 2 * row * n_recv + row * T + 16 * T * K)
+    del partial
+    gathered = torch.empty(R * T, H, dtype=torch.bfloat16, device=dev)
+    res["dense all-gather"] = timed(lambda: ep.ep_dense_allgather(x, gathered, K, E, R), row * T + row * R * T)
+    if R <= 32:
+        res["dense reduce-scatter (2 kernels)"] = timed(
+            lambda: ep.ep_dense_reduce_scatter(idx, out, lay.pair_slot, w, gathered, y, E, R),
+            row * n_pairs + 2 * row * R * T + row * T + 12 * T * K)
+    del gathered, flush
+    return res
+
+
 def host_staged_arms(ep, cfg, x, lay, recv_host, dev, iters=10):
     """Receive buffer in mapped pinned host memory: (i) the dispatch kernel stores straight
     into it; (ii) dispatch packs into device staging and the copy engine moves each rank's
@@ -252,6 +296,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=20)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-graph", action="store_true", help="small workloads: time direct launches, not graph replays")
+    ap.add_argument("--variants", action="store_true",
+                    help="also time the variants around the path (grouping, partial-output combine, dense baseline)")
     ap.add_argument("--seed", type=int, default=0)
     args = ap.parse_args()
     if args.warmup < 3:
@@ -378,6 +424,8 @@ def main():
     if cfg.host_staged:
         host = host_staged_arms(ep, cfg, x, lay, recv, dev)
 
+    variants = time_variants(ep, cfg, idx, w, x, out, lay, n_recv, n_pairs, dev) if args.variants else None
+
     # ---- end to end: one C-ABI call per step, host buffers in, host buffer out
     arena = torch.empty(ep.ep_host_step_arena_bytes(T, K, H, E, R), dtype=torch.uint8, device=dev)
     y_h = torch.empty(T, H, dtype=torch.bfloat16).pin_memory()
@@ -432,6 +480,8 @@ def main():
         "context": "paper reports 2.00x (dispatch) / 1.53x (combine) over NCCL for its dense all-gather/"
                    "reduce-scatter on RTX 4090/5090 PCIe boxes; no number for the routing-aware path",
     }
+    if variants is not None:
+        line["variants"] = variants
     if host is not None:
         line["host_staged"] = host
         link = host["host_link_d2h_GB/s"]

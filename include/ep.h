@@ -171,6 +171,41 @@ int ep_group(const ep_shape_t *shape, const void *recv, int64_t recv_rows, const
              int32_t *status, void *stream);
 
 /*
+ * Combine with partial outputs (Section 2.1, "Communication patterns of dispatch
+ * and combine": the All-to-Allv form returns "partial outputs"): every rank
+ * first sums, per token it received, the weighted outputs of its own experts
+ * into one row of `partial` (receive space, [partial_capacity_rows][H] bf16):
+ *   partial[recv_slot[t][k]] = bf16( fp32 fma chain over the k' (ascending) that
+ *                                    share this receive row of w[t][k']*out[pair_slot[t][k']] )
+ * and the owner adds a token's distinct partial rows in the order of their first k:
+ *   y[t] = bf16( fp32 sum from +0 ).
+ * Two roundings to bf16 instead of one: the result differs from ep_combine by at
+ * most one bf16 half-ulp per partial row. Rows of `partial` no token names are
+ * not touched. Out-of-range slots are skipped with EP_STATUS_CAPACITY.
+ */
+int ep_combine_partial(const ep_shape_t *shape, const void *out, int64_t out_rows,
+                       const int32_t *pair_slot, const int32_t *recv_slot, const float *topk_weights,
+                       void *partial, int64_t partial_capacity_rows, void *y, int32_t *status,
+                       void *stream);
+
+/*
+ * Dense formulation on the same logical ranks (Section 2.1: All-Gather and
+ * Reduce-Scatter, Figure 3; Section 4.2: the volumes 2(N-1)S and N*S), the
+ * baseline the routing-aware path is compared with.
+ * ep_dense_allgather: gathered[r*T + t] = x[t] for every rank r: R*T rows
+ * whatever the routing (gathered is [R*T][H] bf16, device).
+ * ep_dense_reduce_scatter: rank r's dense buffer ordered by source token,
+ *   dense[r*T + t] = bf16( fma chain over the k (ascending) whose expert lives on r ),
+ * +0 where the token has no expert on r, then y[t] = bf16( fp32 sum over
+ * r = 0..R-1 of dense[r*T + t] ). dense is [R*T][H] bf16 (device), fully
+ * written. Needs R <= 32.
+ */
+int ep_dense_allgather(const ep_shape_t *shape, const void *x, void *gathered, void *stream);
+int ep_dense_reduce_scatter(const ep_shape_t *shape, const int32_t *topk_idx, const void *out,
+                            int64_t out_rows, const int32_t *pair_slot, const float *topk_weights,
+                            void *dense, void *y, int32_t *status, void *stream);
+
+/*
  * Host-staged dispatch, copy-engine arm (Section 2.2 and Section 4.3: the DMA
  * engines move contiguous regions only, so routing-dependent rows are first
  * packed by a kernel): ep_dispatch into `staging` (device,

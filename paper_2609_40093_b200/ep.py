@@ -22,6 +22,7 @@ PROBE_READ, PROBE_WRITE, PROBE_COPY, PROBE_MEMCPY = 0, 1, 2, 3
 
 EXPORTS = [
     "ep_layout_workspace_bytes", "ep_layout", "ep_layout_static", "ep_layout_static_scratch_bytes", "ep_dispatch", "ep_combine", "ep_group",
+    "ep_combine_partial", "ep_dense_allgather", "ep_dense_reduce_scatter",
     "ep_dispatch_copy_engine", "ep_host_step_arena_bytes", "ep_host_step", "ep_status",
     "ep_probe_bandwidth", "ep_launch_count", "ep_strerror", "ep_last_cuda_error",
 ]
@@ -66,6 +67,9 @@ def lib() -> ctypes.CDLL:
         L.ep_dispatch.argtypes = [sp, vp, vp, vp, i64, vp, vp]
         L.ep_combine.argtypes = [sp, vp, i64, vp, vp, vp, vp, vp]
         L.ep_group.argtypes = [sp, vp, i64, vp, vp, vp, i64, vp, vp]
+        L.ep_combine_partial.argtypes = [sp, vp, i64, vp, vp, vp, vp, i64, vp, vp, vp]
+        L.ep_dense_allgather.argtypes = [sp, vp, vp, vp]
+        L.ep_dense_reduce_scatter.argtypes = [sp, vp, vp, i64, vp, vp, vp, vp, vp, vp]
         L.ep_dispatch_copy_engine.argtypes = [sp, vp, vp, vp, vp, i64, vp, vp, vp]
         L.ep_host_step_arena_bytes.restype = sz
         L.ep_host_step_arena_bytes.argtypes = [sp]
@@ -76,6 +80,7 @@ def lib() -> ctypes.CDLL:
         L.ep_strerror.restype = ctypes.c_char_p
         L.ep_strerror.argtypes = [i32]
         for name in ["ep_layout", "ep_dispatch", "ep_combine", "ep_group", "ep_dispatch_copy_engine",
+                     "ep_combine_partial", "ep_dense_allgather", "ep_dense_reduce_scatter",
                      "ep_host_step", "ep_status", "ep_probe_bandwidth", "ep_last_cuda_error"]:
             getattr(L, name).restype = i32
         _lib = L
@@ -187,6 +192,32 @@ def ep_group(recv: torch.Tensor, lay: Layout, grouped: torch.Tensor, E: int, R: 
                           _ptr(lay.expert_offsets), _ptr(grouped), grouped.shape[0], _ptr(status), _stream()),
            "ep_group")
     return grouped
+
+
+def ep_combine_partial(out, lay: Layout, topk_weights, partial, y, E: int, R: int, status=None):
+    """Two-stage combine: per-(token, rank) partial rows in the receive space, then their sum."""
+    T, K = lay.pair_slot.shape
+    H = out.shape[1]
+    _check(lib().ep_combine_partial(ctypes.byref(_shape(T, K, H, E, R)), _ptr(out), out.shape[0], _ptr(lay.pair_slot),
+                                    _ptr(lay.recv_slot), _ptr(topk_weights), _ptr(partial), partial.shape[0], _ptr(y),
+                                    _ptr(status), _stream()), "ep_combine_partial")
+    return y
+
+
+def ep_dense_allgather(x, gathered, K: int, E: int, R: int):
+    T, H = x.shape
+    _check(lib().ep_dense_allgather(ctypes.byref(_shape(T, K, H, E, R)), _ptr(x), _ptr(gathered), _stream()),
+           "ep_dense_allgather")
+    return gathered
+
+
+def ep_dense_reduce_scatter(topk_idx, out, pair_slot, topk_weights, dense, y, E: int, R: int, status=None):
+    T, K = topk_idx.shape
+    H = out.shape[1]
+    _check(lib().ep_dense_reduce_scatter(ctypes.byref(_shape(T, K, H, E, R)), _ptr(topk_idx), _ptr(out), out.shape[0],
+                                         _ptr(pair_slot), _ptr(topk_weights), _ptr(dense), _ptr(y), _ptr(status),
+                                         _stream()), "ep_dense_reduce_scatter")
+    return y
 
 
 def ep_dispatch_copy_engine(x, recv_slot, staging, recv_host, E, R, rank_row_offsets_host=None, status=None):
