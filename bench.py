@@ -125,6 +125,36 @@ def host_staged_arms(ep, cfg, x, lay, recv_host, dev, iters=10):
         ep.ep_dispatch_copy_engine(x, lay.recv_slot, staging, recv_host, E, R, rank_row_offsets_host=None)
 
     res = {"host_link_d2h_GB/s": d2h, "host_link_h2d_GB/s": h2d, "rows": n_recv, "bytes_over_link": n_recv * row}
+    # round trip through the bounce buffer on two streams: all uploads then all downloads, or chunk-wise duplex
+    cap = recv_host.shape[0]
+    bounce = torch.empty(2 * cap, cfg.H, dtype=torch.bfloat16).pin_memory()
+    back = torch.empty(cap, cfg.H, dtype=torch.bfloat16, device=dev)
+    up, down = torch.cuda.Stream(), torch.cuda.Stream()
+    offs_host = lay.rank_row_offsets.cpu()
+    torch.cuda.synchronize()
+    trips = {}
+    for duplex, chunks in [(0, 1), (1, 1), (1, 2), (1, 4), (1, 8)]:
+        best = 1e30
+        for rnd in range(iters + 1):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(down)
+            ep.ep_host_roundtrip(x, lay.recv_slot, offs_host, staging, bounce, back, E, R, round=rnd,
+                                 chunks_per_rank=chunks, duplex=bool(duplex), stream_up=up, stream_down=down)
+            b.record(down)
+            torch.cuda.synchronize()
+            best = min(best, a.elapsed_time(b))
+        trips[("duplex" if duplex else "serial") + f", {chunks} chunk(s) per rank"] = {
+            "us": best * 1e3, "GB/s_each_way": n_recv * row / (best * 1e-3) / 1e9, "tokens/s": cfg.T / (best * 1e-3)}
+    # cost of one completion check: the wait kernel on flags that are already posted
+    n_s = max(1, R - 1)
+    flags_dev = torch.full((64,), 3, dtype=torch.int32, device=dev)
+    flags_pin = torch.full((64,), 3, dtype=torch.int32).pin_memory()
+    waits = {}
+    for name, fl in [("flags in device memory", flags_dev), ("flags in pinned host memory", flags_pin)]:
+        waits[name] = {"us": timed(lambda: ep.ep_wait_senders(fl, n_s, 3, 100_000_000)) * 1e3, "senders": n_s}
+
+    res["roundtrip"] = trips
+    res["flag_wait_posted"] = waits
     for name, fn, nbytes in [("kernel_store", arm_kernel, n_recv * row),
                              ("copy_engine_per_rank", arm_copy_known, n_recv * row),
                              ("copy_engine_worst_case", arm_copy_blind, recv_host.shape[0] * row)]:

@@ -58,6 +58,7 @@ typedef enum {
 /* bits of the device status word */
 #define EP_STATUS_BAD_INDEX 1 /* an expert id outside [-1, E) was seen and masked */
 #define EP_STATUS_CAPACITY  2 /* a slot >= the buffer's row capacity was skipped  */
+#define EP_STATUS_TIMEOUT   4 /* ep_wait_senders gave up on at least one sender     */
 
 typedef struct {
     int32_t num_tokens;  /* T */
@@ -219,6 +220,43 @@ int ep_dispatch_copy_engine(const ep_shape_t *shape, const void *x, const int32_
                             const int32_t *rank_row_offsets_host, void *staging,
                             int64_t staging_capacity_rows, void *recv_host, int32_t *status,
                             void *stream);
+
+/*
+ * Host-staged round trip with separate upload and download streams (Section
+ * 4.3: "uploads on one stream, downloads on another", chunked so that both
+ * directions of the host link are busy; Section 4.4: two alternating bounce
+ * buffers). Packs the receive rows into `staging` (device) with the dispatch
+ * kernel on stream_up, copies them chunk by chunk to the bounce buffer
+ * (pinned host, 2 * staging_capacity_rows rows: half `round & 1` is used) and
+ * from there into `recv` (device, same row layout) on stream_down. Each rank's
+ * partition is cut into chunks_per_rank chunks. duplex != 0: a chunk's download
+ * is released by an event right after its upload, so uploads and downloads
+ * overlap; duplex == 0: all uploads, then all downloads. The result is complete
+ * when stream_down is; stream_up first waits for what is queued on stream_down.
+ * rank_row_offsets_host (host, [R+1]) must hold the layout's offsets. Events are
+ * created on first use and kept (no device memory is allocated).
+ */
+int ep_host_roundtrip(const ep_shape_t *shape, const void *x, const int32_t *recv_slot,
+                      const int32_t *rank_row_offsets_host, void *staging, int64_t staging_capacity_rows,
+                      void *bounce_host, int round, void *recv, int chunks_per_rank, int duplex,
+                      int32_t *status, void *stream_up, void *stream_down);
+
+/*
+ * Per-sender completion flags (Section 4.4: the payload stays contiguous and the
+ * flags are stored apart; one thread per sender polls its flag with uncached
+ * loads and pauses between attempts; a flag has a single writer, so no atomics).
+ * ep_wait_senders enqueues a one-CTA kernel whose thread s polls flags[s]
+ * (device memory or mapped pinned host memory) until it reads `epoch`, then
+ * writes `epoch` to arrived[s] (device, may be NULL), the word consumers watch.
+ * Every wait is bounded: after timeout_ns (at most 2 s) the thread gives up,
+ * EP_STATUS_TIMEOUT is OR-ed into *status (device, may be NULL) and the kernel
+ * ends; nothing hangs and later work on the stream still runs. 1 <= num_senders
+ * <= 64. ep_post_flags enqueues the writer side: flags[first..first+n) = epoch,
+ * ordered after all earlier work of its stream.
+ */
+int ep_wait_senders(const uint32_t *flags, int num_senders, uint32_t epoch, uint64_t timeout_ns,
+                    uint32_t *arrived, int32_t *status, void *stream);
+int ep_post_flags(uint32_t *flags, int first_sender, int num_senders, uint32_t epoch, void *stream);
 
 /*
  * One whole step from host buffers: copies x, topk_idx and topk_weights from

@@ -18,11 +18,13 @@ _lib = None
 
 STATUS_BAD_INDEX = 1
 STATUS_CAPACITY = 2
+STATUS_TIMEOUT = 4
 PROBE_READ, PROBE_WRITE, PROBE_COPY, PROBE_MEMCPY = 0, 1, 2, 3
 
 EXPORTS = [
     "ep_layout_workspace_bytes", "ep_layout", "ep_layout_static", "ep_layout_static_scratch_bytes", "ep_dispatch", "ep_combine", "ep_group",
     "ep_combine_partial", "ep_dense_allgather", "ep_dense_reduce_scatter",
+    "ep_host_roundtrip", "ep_wait_senders", "ep_post_flags",
     "ep_dispatch_copy_engine", "ep_host_step_arena_bytes", "ep_host_step", "ep_status",
     "ep_probe_bandwidth", "ep_launch_count", "ep_strerror", "ep_last_cuda_error",
 ]
@@ -70,6 +72,9 @@ def lib() -> ctypes.CDLL:
         L.ep_combine_partial.argtypes = [sp, vp, i64, vp, vp, vp, vp, i64, vp, vp, vp]
         L.ep_dense_allgather.argtypes = [sp, vp, vp, vp]
         L.ep_dense_reduce_scatter.argtypes = [sp, vp, vp, i64, vp, vp, vp, vp, vp, vp]
+        L.ep_host_roundtrip.argtypes = [sp, vp, vp, vp, vp, i64, vp, i32, vp, i32, i32, vp, vp, vp]
+        L.ep_wait_senders.argtypes = [vp, i32, ctypes.c_uint32, ctypes.c_uint64, vp, vp, vp]
+        L.ep_post_flags.argtypes = [vp, i32, i32, ctypes.c_uint32, vp]
         L.ep_dispatch_copy_engine.argtypes = [sp, vp, vp, vp, vp, i64, vp, vp, vp]
         L.ep_host_step_arena_bytes.restype = sz
         L.ep_host_step_arena_bytes.argtypes = [sp]
@@ -81,6 +86,7 @@ def lib() -> ctypes.CDLL:
         L.ep_strerror.argtypes = [i32]
         for name in ["ep_layout", "ep_dispatch", "ep_combine", "ep_group", "ep_dispatch_copy_engine",
                      "ep_combine_partial", "ep_dense_allgather", "ep_dense_reduce_scatter",
+                     "ep_host_roundtrip", "ep_wait_senders", "ep_post_flags",
                      "ep_host_step", "ep_status", "ep_probe_bandwidth", "ep_last_cuda_error"]:
             getattr(L, name).restype = i32
         _lib = L
@@ -228,6 +234,30 @@ def ep_dispatch_copy_engine(x, recv_slot, staging, recv_host, E, R, rank_row_off
                                          _ptr(rank_row_offsets_host), _ptr(staging), staging.shape[0],
                                          _ptr(recv_host), _ptr(status), _stream()), "ep_dispatch_copy_engine")
     return recv_host
+
+
+def ep_host_roundtrip(x, recv_slot, rank_row_offsets_host, staging, bounce_host, recv, E, R, round=0,
+                      chunks_per_rank=1, duplex=True, status=None, stream_up=None, stream_down=None):
+    """Pack -> upload to the pinned bounce buffer -> download into `recv`, on two streams
+    (torch.cuda.Stream objects; default: the current stream for both)."""
+    T, H = x.shape
+    K = recv_slot.shape[1]
+    up = ctypes.c_void_p(stream_up.cuda_stream) if stream_up is not None else _stream()
+    down = ctypes.c_void_p(stream_down.cuda_stream) if stream_down is not None else _stream()
+    _check(lib().ep_host_roundtrip(ctypes.byref(_shape(T, K, H, E, R)), _ptr(x), _ptr(recv_slot),
+                                   _ptr(rank_row_offsets_host), _ptr(staging), staging.shape[0], _ptr(bounce_host),
+                                   int(round), _ptr(recv), int(chunks_per_rank), int(bool(duplex)), _ptr(status), up, down),
+           "ep_host_roundtrip")
+    return recv
+
+
+def ep_wait_senders(flags, num_senders: int, epoch: int, timeout_ns: int, arrived=None, status=None):
+    _check(lib().ep_wait_senders(_ptr(flags), num_senders, epoch, timeout_ns, _ptr(arrived), _ptr(status), _stream()),
+           "ep_wait_senders")
+
+
+def ep_post_flags(flags, first_sender: int, num_senders: int, epoch: int):
+    _check(lib().ep_post_flags(_ptr(flags), first_sender, num_senders, epoch, _stream()), "ep_post_flags")
 
 
 def ep_host_step_arena_bytes(T, K, H, E, R) -> int:
