@@ -35,6 +35,22 @@ NCU_TRAFFIC_BYTES = {("C4", "combine_rows_kernel"): 1037.9e6, ("C4", "dispatch_r
 L2_BYTES = 126e6
 
 
+class L2Flush:
+    """Evicts the working set from the 126 MB L2 between timed steps: writes a 256 MB buffer, then
+    reads a second one, so that L2 ends up holding clean lines of a foreign buffer. (After the write
+    alone, ~126 MB of dirty lines would be written back during the next timed kernel and be charged to it.)"""
+
+    def __init__(self, dev, nbytes=256 << 20):
+        self.w = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+        self.r = torch.zeros(nbytes // 4, dtype=torch.int32, device=dev)
+        self.i = 0
+
+    def __call__(self):
+        self.i += 1
+        self.w.fill_(self.i & 0xff)
+        torch.sum(self.r)
+
+
 def LAUNCHES_PER_STEP(ep, step):
     """Kernels one direct (non-graph) step launches, counted by the library."""
     n0 = ep.ep_launch_count()
@@ -48,7 +64,7 @@ def time_variants(ep, cfg, idx, w, x, out, lay, n_recv, n_pairs, dev, iters=20):
     expanded dispatch, combine with per-rank partial outputs, dense all-gather / reduce-scatter."""
     T, K, H, E, R = cfg.T, cfg.K, cfg.H, cfg.E, cfg.R
     row = 2 * H
-    flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    flush = L2Flush(dev)
     recv = torch.empty(max(1, n_recv), H, dtype=torch.bfloat16, device=dev)
     ep.ep_dispatch(x, lay.recv_slot, recv, E, R)
     y = torch.empty(T, H, dtype=torch.bfloat16, device=dev)
@@ -57,7 +73,7 @@ def time_variants(ep, cfg, idx, w, x, out, lay, n_recv, n_pairs, dev, iters=20):
     def timed(fn, nbytes):
         ts = []
         for _ in range(iters + 2):
-            flush.fill_(1)
+            flush()
             a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             a.record()
             fn()
@@ -411,7 +427,7 @@ def main():
     else:
         # ---- small workloads: L2 is flushed (256 MB written) before every step; each step is timed by its own
         # event pair and the step itself is a CUDA-graph replay, so host launch cost is not what is measured
-        flush = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+        flusher = L2Flush(dev)
         graph = None
         if not args.no_graph:
             side = torch.cuda.Stream()
@@ -426,7 +442,7 @@ def main():
         rep.barrier()
         with ClockSampler(torch.cuda.current_device()) as clocks:
             for i in range(args.steps):
-                flush.fill_(i & 0xff)
+                flusher()
                 s_ev[i].record()
                 graph.replay() if graph is not None else step()
                 e_ev[i].record()
@@ -439,13 +455,14 @@ def main():
         # per-kernel figures from a separate pass of direct launches, each step after a flush
         evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(min(args.steps, 50))]
         for e in evs:
-            flush.fill_(1)
+            flusher()
             step(e)
         torch.cuda.synchronize()
         per = np.array([[e[j].elapsed_time(e[j + 1]) for j in range(3)] for e in evs])
-        l2_note = "step data would fit L2: 256 MB flush write before every timed step, each step timed by its own event pair"
+        l2_note = ("step data would fit L2: before every timed step 256 MB are written and then another 256 MB read "
+                   "(L2 left holding clean foreign lines); each step timed by its own event pair")
         launch_note = "CUDA graph replay of one step" if graph is not None else "direct launches"
-        del flush
+        del flusher
     lay_ms, dis_ms, com_ms = [float(v) for v in per.mean(axis=0)]
     value = world * T * args.steps / (total_ms * 1e-3)
 

@@ -52,9 +52,34 @@ inline int check_shape(const ep_shape_t *s, bool need_hidden)
 
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 
+// Launch with programmatic stream serialisation: the kernel's CTAs may become resident while the
+// previous kernel of the stream is still running; the kernel must execute pdl_wait() before it
+// touches anything an earlier kernel wrote. Stream order is otherwise unchanged.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                              Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 // --- device side ----------------------------------------------------------
 
 #ifdef __CUDACC__
+
+// Blocks until every kernel this one depends on has completed and its writes are visible.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// Lets the next kernel of the stream become resident (it still waits in its own pdl_wait()).
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 __device__ __forceinline__ unsigned lanemask_lt()
 {

@@ -144,11 +144,15 @@ __device__ __forceinline__ unsigned long long token_rank_mask(const LayoutArgs &
     return mask;
 }
 
-// One warp counts its tile into hist[bins] (shared memory, this warp's own).
+// One warp counts its tile into hist[bins]. kShared == false: hist is this warp's own and is
+// zeroed here; kShared == true: hist is one histogram for the whole CTA, zeroed by the caller.
+template <bool kShared>
 __device__ __forceinline__ void count_tile(const LayoutArgs &a, int32_t *hist, int32_t *ids, int tile, int lane)
 {
-    for (int b = lane; b < a.bins; b += 32) hist[b] = 0;
-    __syncwarp();
+    if (!kShared) {
+        for (int b = lane; b < a.bins; b += 32) hist[b] = 0;
+        __syncwarp();
+    }
     if (tile >= a.n_tiles) return;
     const int t0 = tile * a.tile_tokens;
     const int t1 = min(a.T, t0 + a.tile_tokens);
@@ -163,7 +167,10 @@ __device__ __forceinline__ void count_tile(const LayoutArgs &a, int32_t *hist, i
         const unsigned long long mask = token_rank_mask(a, ids, lane);   // rank hits: token per lane, ballot per rank
         for (int r = 0; r < a.R; ++r) {
             const unsigned b = __ballot_sync(kFullMask, (mask >> r) & 1ull);
-            if (lane == 0) hist[a.E + r] += __popc(b);
+            if (lane == 0 && b) {
+                if (kShared) atomicAdd(hist + a.E + r, __popc(b));
+                else hist[a.E + r] += __popc(b);
+            }
         }
         __syncwarp();
     }
@@ -209,18 +216,16 @@ __device__ void block_exclusive_scan_smem(int32_t *v, int n, int32_t *sh)
 // ---------------------------------------------------------------- global form, first kernel
 __global__ void __launch_bounds__(kMaxWarps * 32) layout_cta_count_kernel(LayoutArgs a)
 {
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");   // the main kernel may start its own counting now
+    pdl_trigger();                                                    // the main kernel may start its own counting now
     extern __shared__ int32_t smem[];
     const int warps = blockDim.x >> 5, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int pw = a.bins + kMaxRanks + 64 * a.K;
-    count_tile(a, smem + warp * pw, smem + warp * pw + a.bins + kMaxRanks + 32 * a.K, blockIdx.x * warps + warp, lane);
+    // one histogram for the CTA (first `bins` words), per-warp id staging behind it
+    for (int b = threadIdx.x; b < a.bins; b += blockDim.x) smem[b] = 0;
+    __syncthreads();
+    count_tile<true>(a, smem, smem + a.bins + warp * 32 * a.K, blockIdx.x * warps + warp, lane);
     __syncthreads();
     int32_t *dst = a.cta_part + (size_t)blockIdx.x * a.bins;
-    for (int b = threadIdx.x; b < a.bins; b += blockDim.x) {
-        int32_t sum = 0;
-        for (int w = 0; w < warps; ++w) sum += smem[w * pw + b];
-        dst[b] = sum;
-    }
+    for (int b = threadIdx.x; b < a.bins; b += blockDim.x) dst[b] = smem[b];
 }
 
 // ---------------------------------------------------------------- main kernel
@@ -234,33 +239,26 @@ __global__ void __launch_bounds__(kMaxWarpsSingle * 32) layout_assign_kernel(Lay
     unsigned *bal = reinterpret_cast<unsigned *>(run + a.bins);      // [R] ballots of the current 32 tokens
     int32_t *slot_s = run + a.bins + kMaxRanks;                      // [32*K] receive slots of the current 32 tokens
     int32_t *ids = slot_s + 32 * a.K;                                // [32*K] expert ids of the current 32 tokens
-    int32_t *tot_e = smem + warps * pw;                              // [E+1] expert totals -> offsets
-    int32_t *tot_r = tot_e + a.E + 1;                                // [R+1] rank totals -> offsets
-    int32_t *pre = tot_r + a.R + 1;                                  // [bins] count in earlier CTAs
+    int32_t *tot = smem + warps * pw;                                // [E+R+1] totals -> one scan: experts, then ranks
+    int32_t *pre = tot + a.bins + 1;                                 // [bins] count in earlier CTAs
     int32_t *cta_tot = pre + a.bins;                                 // [bins] this CTA's totals (peers read it)
     int32_t *sh = cta_tot + a.bins;                                  // [32] scan scratch
     const int tile = blockIdx.x * warps + warp;
     const unsigned lt = lanemask_lt();
 
     EP_STAMP(0);
-    count_tile(a, run, ids, tile, lane);
+    count_tile<false>(a, run, ids, tile, lane);
     __syncthreads();
     EP_STAMP(1);
-    // per bin: exclusive prefix over this CTA's warps (in place) and the CTA total
-    for (int b = threadIdx.x; b < a.bins; b += blockDim.x) {
+    for (int b = threadIdx.x; b < a.bins; b += blockDim.x) {         // this CTA's total per bin
         int32_t mine = 0;
-        for (int w = 0; w < warps; ++w) {
-            const int32_t v = smem[w * pw + b];
-            smem[w * pw + b] = mine;
-            mine += v;
-        }
+        for (int w = 0; w < warps; ++w) mine += smem[w * pw + b];
         cta_tot[b] = mine;
     }
     if (a.mode == kModeCluster) cg::this_cluster().sync();           // every peer's cta_tot is written
-    else if (a.mode == kModeGlobal) asm volatile("griddepcontrol.wait;" ::: "memory");   // cta_part is complete and visible
-    else __syncthreads();
+    else if (a.mode == kModeGlobal) pdl_wait();                      // cta_part is complete and visible
     EP_STAMP(2);
-    // per bin: count in earlier CTAs and grand total
+    // per bin: count in earlier CTAs and grand total (each thread reads the cta_tot entries it wrote itself)
     for (int b = threadIdx.x; b < a.bins; b += blockDim.x) {
         int32_t before = 0, total = 0;
         if (a.mode == kModeCluster) {
@@ -282,8 +280,7 @@ __global__ void __launch_bounds__(kMaxWarpsSingle * 32) layout_assign_kernel(Lay
             total = cta_tot[b];
         }
         pre[b] = before;
-        if (b < a.E) tot_e[b] = total;
-        else if (b < nb) tot_r[b - a.E] = total;
+        if (b < nb) tot[b] = total;
         if (blockIdx.x == 0) {
             if (b < a.E) a.out.expert_counts[b] = total;
             else if (b < nb) a.out.rank_rows[b - a.E] = total;
@@ -293,16 +290,23 @@ __global__ void __launch_bounds__(kMaxWarpsSingle * 32) layout_assign_kernel(Lay
     if (a.mode == kModeCluster) cg::this_cluster().sync();           // peers are done with this CTA's shared memory
     else __syncthreads();
     EP_STAMP(3);
-    block_exclusive_scan_smem(tot_e, a.E, sh);
-    block_exclusive_scan_smem(tot_r, a.R, sh);
+    // one exclusive scan over [experts | ranks]: S[e] = expert offset, S[E + r] - S[E] = rank row offset
+    block_exclusive_scan_smem(tot, nb, sh);
+    const int32_t n_pairs = tot[a.E];
     if (blockIdx.x == 0) {
-        for (int e = threadIdx.x; e <= a.E; e += blockDim.x) a.out.expert_offsets[e] = tot_e[e];
-        for (int r = threadIdx.x; r <= a.R; r += blockDim.x) a.out.rank_row_offsets[r] = tot_r[r];
-        for (int r = threadIdx.x; r < a.R; r += blockDim.x) a.out.src_row_offsets[r * (a.R + 1) + a.R] = tot_r[r + 1];
+        for (int e = threadIdx.x; e <= a.E; e += blockDim.x) a.out.expert_offsets[e] = tot[e];
+        for (int r = threadIdx.x; r <= a.R; r += blockDim.x) a.out.rank_row_offsets[r] = tot[a.E + r] - n_pairs;
+        for (int r = threadIdx.x; r < a.R; r += blockDim.x)
+            a.out.src_row_offsets[r * (a.R + 1) + a.R] = tot[a.E + r + 1] - n_pairs;
     }
+    // next free slot of every bin for every warp: offset + earlier CTAs + earlier warps of this CTA
     for (int b = threadIdx.x; b < nb; b += blockDim.x) {
-        const int32_t base = pre[b] + (b < a.E ? tot_e[b] : tot_r[b - a.E]);
-        for (int w = 0; w < warps; ++w) smem[w * pw + b] += base;
+        int32_t running = pre[b] + (b < a.E ? tot[b] : tot[b] - n_pairs);
+        for (int w = 0; w < warps; ++w) {
+            const int32_t v = smem[w * pw + b];
+            smem[w * pw + b] = running;
+            running += v;
+        }
     }
     __syncthreads();
     EP_STAMP(4);

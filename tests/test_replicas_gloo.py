@@ -17,12 +17,18 @@ def _torchrun(script_args, port):
 
 
 def _json_lines(text):
-    out = []
-    for line in text.splitlines():
-        line = line.strip()
-        if line.startswith("{") and line.endswith("}"):
-            out.append(json.loads(line))
-    return out
+    """Every JSON object in the text (two ranks may write to the same line)."""
+    out, dec, i = [], json.JSONDecoder(), 0
+    while True:
+        i = text.find("{", i)
+        if i < 0:
+            return out
+        try:
+            obj, end = dec.raw_decode(text, i)
+            out.append(obj)
+            i = end
+        except json.JSONDecodeError:
+            i += 1
 
 
 def test_two_gloo_ranks_run_independent_replicas():
