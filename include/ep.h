@@ -272,6 +272,22 @@ int ep_host_step(const ep_shape_t *shape, const void *x_host, const int32_t *top
                  const float *topk_weights_host, void *y_host, int32_t *status_host, void *arena,
                  size_t arena_bytes, void *stream);
 
+/*
+ * The same step with the host link used in both directions at once (Section 4.3:
+ * uploads and downloads on separate streams, cut into chunks): the tokens are
+ * cut into `chunks` contiguous chunks; chunk c's rows are uploaded on stream_in
+ * while chunk c-1 runs dispatch, local grouping and combine on stream_compute
+ * and chunk c-2's result is downloaded on stream_out (layout runs once, on the
+ * whole routing table, before the first chunk). Results are identical to
+ * ep_host_step. Complete when stream_out is. The three streams must differ for
+ * any overlap; the arena may be reused by the next call without synchronising
+ * (the call orders itself after the previous one). 1 <= chunks <= 256.
+ */
+int ep_host_step_pipelined(const ep_shape_t *shape, const void *x_host, const int32_t *topk_idx_host,
+                           const float *topk_weights_host, void *y_host, int32_t *status_host, void *arena,
+                           size_t arena_bytes, int chunks, void *stream_in, void *stream_compute,
+                           void *stream_out);
+
 /* Reads a device status word: copies it to *status_host and SYNCHRONISES the stream. */
 int ep_status(const int32_t *status_dev, void *stream, int32_t *status_host);
 

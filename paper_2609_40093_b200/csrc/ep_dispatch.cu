@@ -126,7 +126,58 @@ group_rows_kernel(const uint4 *__restrict__ recv, long long recv_rows, const int
     }
 }
 
+// dst[dst_slot[i]] = src[src_slot[i]] for i in [0, n): the local grouping written pair by pair, so that
+// it can run on any contiguous range of pairs (a token chunk) as soon as that chunk's rows exist.
+template <int U>
+__global__ void __launch_bounds__(U >= 8 ? 256 : (U == 4 ? 512 : 1024))
+permute_rows_kernel(const uint4 *__restrict__ src, long long src_rows, const int32_t *__restrict__ src_slot,
+                    uint4 *dst, long long dst_rows, const int32_t *__restrict__ dst_slot, long long n,
+                    int vec_per_row, int G, int32_t *status)
+{
+    const int g = threadIdx.x % G;
+    const long long i = (long long)blockIdx.x * (blockDim.x / G) + threadIdx.x / G;
+    if (i >= n) return;
+    const int32_t s = __ldg(src_slot + i), d = __ldg(dst_slot + i);
+    if (s < 0 || d < 0) return;                           // masked pair
+    if (s >= src_rows || d >= dst_rows) {
+        if (g == 0) flag_status(status, EP_STATUS_CAPACITY);
+        return;
+    }
+    const uint4 *from = src + (size_t)s * vec_per_row;
+    uint4 *to = dst + (size_t)d * vec_per_row;
+    for (int v0 = g; v0 < vec_per_row; v0 += G * U) {
+        uint4 buf[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int v = v0 + u * G;
+            if (v < vec_per_row) buf[u] = ld_stream(from + v);
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int v = v0 + u * G;
+            if (v < vec_per_row) st_stream(to + v, buf[u]);
+        }
+    }
+}
+
 }  // namespace
+
+int launch_permute(int hidden, const void *src, int64_t src_rows, const int32_t *src_slot, void *dst,
+                   int64_t dst_rows, const int32_t *dst_slot, int64_t n, int32_t *status, cudaStream_t stream)
+{
+    if (n <= 0) return EP_OK;
+    const int vpr = hidden / 8;
+    const RowPlan p = plan_rows(vpr, "EP_TUNE_GROUP");
+    const unsigned grid = (unsigned)((n + p.rows_per_block - 1) / p.rows_per_block);
+    const uint4 *s4 = static_cast<const uint4 *>(src);
+    uint4 *d4 = static_cast<uint4 *>(dst);
+    if (p.U == 1)
+        permute_rows_kernel<1><<<grid, p.block, 0, stream>>>(s4, src_rows, src_slot, d4, dst_rows, dst_slot, n, vpr, p.G, status);
+    else
+        permute_rows_kernel<2><<<grid, p.block, 0, stream>>>(s4, src_rows, src_slot, d4, dst_rows, dst_slot, n, vpr, p.G, status);
+    EP_LAUNCH_CHECK(1);
+    return EP_OK;
+}
 
 int launch_dispatch(const ep_shape_t &s, const void *x, const int32_t *recv_slot, void *recv,
                     int64_t capacity_rows, int32_t *status, cudaStream_t stream)

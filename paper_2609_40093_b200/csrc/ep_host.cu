@@ -2,6 +2,7 @@
 // host-staged dispatch, the whole step from host buffers, the status read-back,
 // bandwidth probes, and the error / launch bookkeeping.
 #include <atomic>
+#include <mutex>
 
 #include "ep_common.cuh"
 
@@ -14,11 +15,36 @@ int launch_group(const ep_shape_t &s, const void *recv, int64_t recv_rows, const
                  cudaStream_t stream);
 int launch_combine(const ep_shape_t &s, const void *out, int64_t out_rows, const int32_t *slot,
                    const float *weights, void *y, int32_t *status, cudaStream_t stream);
+int launch_permute(int hidden, const void *src, int64_t src_rows, const int32_t *src_slot, void *dst,
+                   int64_t dst_rows, const int32_t *dst_slot, int64_t n, int32_t *status, cudaStream_t stream);
 
 namespace {
 std::atomic<int> g_last_cuda_error{0};
 std::atomic<long long> g_launches{0};
 }  // namespace
+
+// Timing-free events for cross-stream ordering: created on first use, kept for the life of the process.
+namespace {
+constexpr int kEventPool = 1024;
+cudaEvent_t g_events[64][kEventPool];
+int g_events_ready[64] = {};
+std::mutex g_event_mutex;
+}  // namespace
+
+int order_events(cudaEvent_t **pool, int need)
+{
+    if (need > kEventPool) return EP_ERR_INVALID_ARG;
+    int dev = 0;
+    EP_CUDA_TRY(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return EP_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lock(g_event_mutex);
+    while (g_events_ready[dev] < need) {
+        EP_CUDA_TRY(cudaEventCreateWithFlags(&g_events[dev][g_events_ready[dev]], cudaEventDisableTiming));
+        ++g_events_ready[dev];
+    }
+    *pool = g_events[dev];
+    return EP_OK;
+}
 
 void note_cuda_error(cudaError_t e) { g_last_cuda_error.store((int)e); }
 void count_launches(int n) { g_launches.fetch_add(n); }
@@ -179,6 +205,67 @@ extern "C" int ep_host_step(const ep_shape_t *shape, const void *x_host, const i
     EP_CUDA_TRY(cudaMemcpyAsync(y_host, b.y, T * H * 2, cudaMemcpyDeviceToHost, stream));
     if (status_host)
         EP_CUDA_TRY(cudaMemcpyAsync(status_host, b.lay.status, sizeof(int32_t), cudaMemcpyDeviceToHost, stream));
+    return EP_OK;
+}
+
+extern "C" int ep_host_step_pipelined(const ep_shape_t *shape, const void *x_host, const int32_t *topk_idx_host,
+                                      const float *topk_weights_host, void *y_host, int32_t *status_host,
+                                      void *arena, size_t arena_bytes, int chunks, void *stream_in_,
+                                      void *stream_compute_, void *stream_out_)
+{
+    using namespace ep;
+    int rc = check_shape(shape, true);
+    if (rc != EP_OK) return rc;
+    if (!arena) return EP_ERR_NULL;
+    if ((reinterpret_cast<uintptr_t>(arena) & 255u) != 0 || chunks < 1 || chunks > 256) return EP_ERR_INVALID_ARG;
+    const StepBuffers b = carve_step(*shape, arena);
+    if (arena_bytes < b.total) return EP_ERR_CAPACITY;
+    if (shape->num_tokens == 0) return EP_OK;
+    if (!x_host || !topk_idx_host || !topk_weights_host || !y_host) return EP_ERR_NULL;
+    cudaStream_t in = static_cast<cudaStream_t>(stream_in_), comp = static_cast<cudaStream_t>(stream_compute_),
+                 outs = static_cast<cudaStream_t>(stream_out_);
+    cudaEvent_t *ev = nullptr;
+    rc = order_events(&ev, 2 * chunks + 3);
+    if (rc != EP_OK) return rc;
+    const size_t T = shape->num_tokens, K = shape->top_k, H = shape->hidden;
+    // the arena is reused from step to step: uploads wait for the previous step's kernels, and the
+    // kernels for the previous step's downloads of y
+    EP_CUDA_TRY(cudaEventRecord(ev[0], comp));
+    EP_CUDA_TRY(cudaStreamWaitEvent(in, ev[0], 0));
+    EP_CUDA_TRY(cudaEventRecord(ev[1], outs));
+    EP_CUDA_TRY(cudaStreamWaitEvent(comp, ev[1], 0));
+    EP_CUDA_TRY(cudaMemcpyAsync(b.idx, topk_idx_host, T * K * sizeof(int32_t), cudaMemcpyHostToDevice, in));
+    EP_CUDA_TRY(cudaMemcpyAsync(b.w, topk_weights_host, T * K * sizeof(float), cudaMemcpyHostToDevice, in));
+    EP_CUDA_TRY(cudaEventRecord(ev[2], in));
+    EP_CUDA_TRY(cudaStreamWaitEvent(comp, ev[2], 0));
+    rc = ep_layout(shape, b.idx, &b.lay, b.workspace, b.workspace_bytes, comp);
+    if (rc != EP_OK) return rc;
+    for (int c = 0; c < chunks; ++c) {
+        const size_t t0 = T * c / chunks, t1 = T * (c + 1) / chunks, n = t1 - t0;
+        if (n == 0) continue;
+        ep_shape_t part = *shape;
+        part.num_tokens = (int32_t)n;
+        // upload this chunk of x while earlier chunks are being processed and downloaded
+        EP_CUDA_TRY(cudaMemcpyAsync(b.x + t0 * H, static_cast<const uint16_t *>(x_host) + t0 * H, n * H * 2,
+                                    cudaMemcpyHostToDevice, in));
+        EP_CUDA_TRY(cudaEventRecord(ev[3 + 2 * c], in));
+        EP_CUDA_TRY(cudaStreamWaitEvent(comp, ev[3 + 2 * c], 0));
+        rc = launch_dispatch(part, b.x + t0 * H, b.lay.recv_slot + t0 * K, b.recv, b.recv_rows, b.lay.status, comp);
+        if (rc != EP_OK) return rc;
+        // identity expert: the chunk's pair rows are its receive rows
+        rc = launch_permute(shape->hidden, b.recv, b.recv_rows, b.lay.recv_slot + t0 * K, b.grouped, b.pair_rows,
+                            b.lay.pair_slot + t0 * K, (int64_t)(n * K), b.lay.status, comp);
+        if (rc != EP_OK) return rc;
+        rc = launch_combine(part, b.grouped, b.pair_rows, b.lay.pair_slot + t0 * K, b.w + t0 * K, b.y + t0 * H,
+                            b.lay.status, comp);
+        if (rc != EP_OK) return rc;
+        EP_CUDA_TRY(cudaEventRecord(ev[4 + 2 * c], comp));
+        EP_CUDA_TRY(cudaStreamWaitEvent(outs, ev[4 + 2 * c], 0));
+        EP_CUDA_TRY(cudaMemcpyAsync(static_cast<uint16_t *>(y_host) + t0 * H, b.y + t0 * H, n * H * 2,
+                                    cudaMemcpyDeviceToHost, outs));
+    }
+    if (status_host)
+        EP_CUDA_TRY(cudaMemcpyAsync(status_host, b.lay.status, sizeof(int32_t), cudaMemcpyDeviceToHost, outs));
     return EP_OK;
 }
 

@@ -9,14 +9,13 @@
 // on %globaltimer and an iteration count): when the bound is hit the thread gives
 // up, sets EP_STATUS_TIMEOUT and the kernel returns, so the stream and the context
 // stay usable.
-#include <mutex>
-
 #include "ep_common.cuh"
 
 namespace ep {
 
 int launch_dispatch(const ep_shape_t &s, const void *x, const int32_t *recv_slot, void *recv,
                     int64_t capacity_rows, int32_t *status, cudaStream_t stream);
+int order_events(cudaEvent_t **pool, int need);
 
 namespace {
 
@@ -71,27 +70,6 @@ __global__ void post_flags_kernel(uint32_t *flags, int first, int n, uint32_t ep
     asm volatile("st.volatile.global.u32 [%0], %1;" ::"l"(flags + first + s), "r"(epoch) : "memory");
 }
 
-// events for the round trip: created on first use, kept for the life of the process
-constexpr int kEventPool = 1024;
-cudaEvent_t g_events[64][kEventPool];
-int g_events_ready[64] = {};
-std::mutex g_event_mutex;
-
-int round_trip_events(cudaEvent_t **pool, int need)
-{
-    if (need > kEventPool) return EP_ERR_INVALID_ARG;
-    int dev = 0;
-    EP_CUDA_TRY(cudaGetDevice(&dev));
-    if (dev < 0 || dev >= 64) return EP_ERR_INVALID_ARG;
-    std::lock_guard<std::mutex> lock(g_event_mutex);
-    while (g_events_ready[dev] < need) {
-        EP_CUDA_TRY(cudaEventCreateWithFlags(&g_events[dev][g_events_ready[dev]], cudaEventDisableTiming));
-        ++g_events_ready[dev];
-    }
-    *pool = g_events[dev];
-    return EP_OK;
-}
-
 }  // namespace
 }  // namespace ep
 
@@ -137,7 +115,7 @@ extern "C" int ep_host_roundtrip(const ep_shape_t *shape, const void *x, const i
         if (rank_row_offsets_host[r + 1] < rank_row_offsets_host[r]) return EP_ERR_INVALID_ARG;
     cudaStream_t up = static_cast<cudaStream_t>(stream_up_), down = static_cast<cudaStream_t>(stream_down_);
     cudaEvent_t *ev = nullptr;
-    rc = round_trip_events(&ev, R * chunks_per_rank + 2);
+    rc = order_events(&ev, R * chunks_per_rank + 2);
     if (rc != EP_OK) return rc;
     const size_t row_bytes = (size_t)shape->hidden * 2;
     // two bounce buffers alternate by round, so a buffer is reused only every other round

@@ -24,7 +24,7 @@ PROBE_READ, PROBE_WRITE, PROBE_COPY, PROBE_MEMCPY = 0, 1, 2, 3
 EXPORTS = [
     "ep_layout_workspace_bytes", "ep_layout", "ep_layout_static", "ep_layout_static_scratch_bytes", "ep_dispatch", "ep_combine", "ep_group",
     "ep_combine_partial", "ep_dense_allgather", "ep_dense_reduce_scatter",
-    "ep_host_roundtrip", "ep_wait_senders", "ep_post_flags",
+    "ep_host_roundtrip", "ep_wait_senders", "ep_post_flags", "ep_host_step_pipelined",
     "ep_dispatch_copy_engine", "ep_host_step_arena_bytes", "ep_host_step", "ep_status",
     "ep_probe_bandwidth", "ep_launch_count", "ep_strerror", "ep_last_cuda_error",
 ]
@@ -79,6 +79,8 @@ def lib() -> ctypes.CDLL:
         L.ep_host_step_arena_bytes.restype = sz
         L.ep_host_step_arena_bytes.argtypes = [sp]
         L.ep_host_step.argtypes = [sp, vp, vp, vp, vp, vp, vp, sz, vp]
+        L.ep_host_step_pipelined.argtypes = [sp, vp, vp, vp, vp, vp, vp, sz, i32, vp, vp, vp]
+        L.ep_host_step_pipelined.restype = i32
         L.ep_status.argtypes = [vp, vp, vp]
         L.ep_probe_bandwidth.argtypes = [i32, vp, vp, sz, i32, vp, ctypes.POINTER(ctypes.c_double)]
         L.ep_launch_count.restype = i64
@@ -271,6 +273,19 @@ def ep_host_step(x_host, topk_idx_host, topk_weights_host, y_host, arena, E, R, 
     _check(lib().ep_host_step(ctypes.byref(_shape(T, K, H, E, R)), _ptr(x_host), _ptr(topk_idx_host),
                               _ptr(topk_weights_host), _ptr(y_host), _ptr(status_host), _ptr(arena), arena.numel(),
                               _stream()), "ep_host_step")
+    return y_host
+
+
+def ep_host_step_pipelined(x_host, topk_idx_host, topk_weights_host, y_host, arena, E, R, chunks, stream_in,
+                           stream_compute, stream_out, status_host=None):
+    """`ep_host_step` with uploads, kernels and downloads of token chunks overlapping on three streams."""
+    T, H = x_host.shape
+    K = topk_idx_host.shape[1]
+    _check(lib().ep_host_step_pipelined(ctypes.byref(_shape(T, K, H, E, R)), _ptr(x_host), _ptr(topk_idx_host),
+                                        _ptr(topk_weights_host), _ptr(y_host), _ptr(status_host), _ptr(arena),
+                                        arena.numel(), int(chunks), ctypes.c_void_p(stream_in.cuda_stream),
+                                        ctypes.c_void_p(stream_compute.cuda_stream),
+                                        ctypes.c_void_p(stream_out.cuda_stream)), "ep_host_step_pipelined")
     return y_host
 
 

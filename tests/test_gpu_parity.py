@@ -202,6 +202,34 @@ def test_host_step_matches_oracle():
     np.testing.assert_array_equal(yh.view(torch.int16).numpy().view(np.uint16), want)
 
 
+@pytest.mark.parametrize("chunks", [1, 3, 8])
+def test_pipelined_host_step_matches_oracle(chunks):
+    """Uploads, kernels and downloads of token chunks overlap on three streams; the result is the
+    same as the one-stream step, also when two calls follow each other without a synchronisation."""
+    cfg = inputs.CONFIGS["C3"]
+    ref_y = []
+    hosts = []
+    for seed in (0, 1):
+        d = inputs.make_inputs(cfg, seed)
+        idx, w, x = d["topk_idx"], d["topk_weights"], d["x"]
+        ref = oracle.layout(idx, cfg.E, cfg.R)
+        recv = oracle.dispatch(x, ref.recv_slot, ref.n_recv)
+        ref_y.append(oracle.combine_f32(recv[ref.pair_row], ref.pair_slot, w))
+        hosts.append((torch.from_numpy(x.view(np.int16)).view(torch.bfloat16).pin_memory(),
+                      torch.from_numpy(idx).pin_memory(), torch.from_numpy(w).pin_memory(),
+                      torch.zeros(cfg.T, cfg.H, dtype=torch.bfloat16).pin_memory(),
+                      torch.full((1,), -1, dtype=torch.int32).pin_memory()))
+    arena = torch.empty(ep.ep_host_step_arena_bytes(cfg.T, cfg.K, cfg.H, cfg.E, cfg.R), dtype=torch.uint8, device="cuda")
+    s_in, s_comp, s_out = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    for xh, ih, wh, yh, sh in hosts:                    # back to back, same arena, no synchronisation between
+        ep.ep_host_step_pipelined(xh, ih, wh, yh, arena, cfg.E, cfg.R, chunks, s_in, s_comp, s_out, status_host=sh)
+    torch.cuda.synchronize()
+    for (xh, ih, wh, yh, sh), want in zip(hosts, ref_y):
+        assert int(sh[0]) == 0
+        np.testing.assert_array_equal(yh.view(torch.int16).numpy().view(np.uint16), want)
+
+
 def test_host_staged_dispatch_both_arms():
     """Receive buffer in mapped pinned host memory: kernel stores and the copy-engine arm."""
     cfg = inputs.CONFIGS["C5"]
