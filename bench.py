@@ -373,10 +373,8 @@ def main():
     w_h = torch.from_numpy(d["topk_weights"]).pin_memory()
     x_h = torch.from_numpy(d["x"].view(np.int16)).view(torch.bfloat16).pin_memory()
     idx, w, x = idx_h.to(dev), w_h.to(dev), x_h.to(dev)
-    gen = torch.Generator(device=dev).manual_seed(1000 * args.seed + rank)
-    out = torch.empty(T * K, H, dtype=torch.bfloat16, device=dev)     # expert outputs, pair space
-    for r0 in range(0, T * K, 8192):
-        out[r0:r0 + 8192] = torch.randn(min(8192, T * K - r0), H, generator=gen, device=dev, dtype=torch.float32)
+    out_h = inputs.make_out(rcfg, T * K, args.seed)                   # expert outputs, pair space (seeded, host)
+    out = torch.from_numpy(out_h.view(np.int16)).view(torch.bfloat16).to(dev)
     lay = ep.alloc_layout(T, K, E, R, device=dev)
     ws = torch.empty(max(16, ep.ep_layout_workspace_bytes(T, K, E, R)), dtype=torch.uint8, device=dev)
     recv = torch.empty(T * min(K, R), H, dtype=torch.bfloat16, device=dev)
@@ -546,7 +544,6 @@ def main():
                                      "peak_kind": "cudaMemcpyAsync D2H probe, 256 MB pinned, same run", "unit": "GB/s",
                                      "frac": host["kernel_store"]["GB/s"] / link, "traffic": None}
     if not args.no_cpu_baseline:
-        out_h = out.view(torch.int16).cpu().numpy().view(np.uint16)
         v, n, el = time_oracle(cfg, d["topk_idx"], d["topk_weights"], d["x"], out_h, min_seconds=10.0, max_steps=20)
         line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle",
                                 "sample": f"{n} whole step(s) of the same {cfg.name} batch in {el:.1f} s, one thread",

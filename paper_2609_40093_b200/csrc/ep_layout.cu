@@ -318,7 +318,8 @@ __global__ void __launch_bounds__(kMaxWarpsSingle * 32) layout_assign_kernel(Lay
     for (int tb = t0; tb < t1; tb += 32) {
         const int t = tb + lane;
         const bool live = t < t1;
-        const int n_items = stage_group(a, ids, tb, t1, lane);
+        // a tile of one 32-token group still has its ids staged from the counting phase
+        const int n_items = a.tile_tokens == 32 ? (min(t1, tb + 32) - tb) * a.K : stage_group(a, ids, tb, t1, lane);
         // --- receive rows: which of these 32 tokens hit which rank
         const unsigned long long mask = token_rank_mask(a, ids, lane);
         for (int r = 0; r < a.R; ++r) {
