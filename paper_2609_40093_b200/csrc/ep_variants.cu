@@ -51,7 +51,7 @@ GroupPlan plan_group(int vec_per_row)
 // receive row in the routed form, the destination rank in the dense form); for
 // every part, dst[row(part)] = bf16( fma chain over the part's k in ascending order ).
 // Dense form: parts are the ranks 0..R-1, row = r*T + t, empty parts write +0.
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, 3)
 reduce_to_rows_kernel(const uint4 *__restrict__ out, long long out_rows, const int32_t *__restrict__ pair_slot,
                       const int32_t *__restrict__ recv_slot, const int32_t *__restrict__ topk_idx,
                       const float *__restrict__ weights, uint4 *dst, long long dst_rows, int T, int K, int E, int R,
@@ -176,7 +176,7 @@ reduce_to_rows_kernel(const uint4 *__restrict__ out, long long out_rows, const i
 // Stage 2: y[t] = bf16( fp32 sum from +0 of the rows the token names ). Routed form: the
 // token's distinct receive rows in the order of their first k (slot table with
 // duplicates). Dense form (slot == nullptr): rows r*T + t for r = 0..R-1.
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(256, 4)
 sum_rows_kernel(const uint4 *__restrict__ src, long long src_rows, const int32_t *__restrict__ slot,
                 uint4 *__restrict__ y, int T, int K, int vec_per_row, int G, int32_t *status)
 {
