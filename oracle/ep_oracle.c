@@ -33,15 +33,16 @@
  *   - combine: fp32 fused multiply-add chain from +0 in ascending k, one
  *     round-to-nearest-even narrowing to bf16 at the end
  *
- * Parity pins (tests, CPU only): brute-force evaluation of the set expressions
- * on tiny inputs, numpy bincount / cumsum / stable argsort on every config,
- * closed forms (R = 1, E = R, one-hot weights, K = 1, constant rows), the
- * invariants (counts sum to the number of valid pairs; receive rows = number of
- * distinct (token, rank); rows <= T*min(K,R); identity expert with weights
- * summing to 1 returns x), the constructed case of the paper's Figure 3 caption,
- * and an exact-rational evaluation of the combine sum. The paper prints no
- * worked values for this path: parity is unpinned by the paper itself and pinned
- * by the mathematics only.
+ * Pins (tests, CPU only). The paper prints no worked values for this path, so
+ * every function here is pinned by the mathematics instead: brute-force
+ * evaluation of the set expressions on tiny inputs; numpy bincount / cumsum /
+ * stable argsort on every config; closed forms (R = 1, E = R, one-hot weights,
+ * K = 1, constant rows); the invariants (counts sum to the number of valid
+ * pairs; receive rows = number of distinct (token, rank); rows <= T*min(K,R);
+ * identity expert with weights summing to 1 returns x); the constructed case of
+ * the paper's Figure 3 caption; exact-rational evaluation of the combine chains
+ * with explicit roundings; and, for the dense formulation, the paper's volume
+ * formulas of Section 4.2.
  */
 #include <math.h>
 #include <stdint.h>

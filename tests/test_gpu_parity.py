@@ -150,6 +150,19 @@ def test_identity_expert_roundtrip_and_one_hot_weights():
         np.testing.assert_array_equal(host_bits(y), x)
 
 
+def test_combine_uses_fused_multiply_add():
+    """acc = -c, then w*v = c + c*2^-23: one rounding leaves c*2^-23, a rounded product 2^-23."""
+    c = 1.0078125                                           # 1 + 2^-7, a bf16 number
+    out = inputs.to_bf16_bits(np.full((2, 64), c, dtype=np.float32))
+    slot = np.tile(np.array([[0, 1]], dtype=np.int32), (4, 1))
+    w = np.tile(np.array([[-1.0, 1.0 + 2.0 ** -23]], dtype=np.float32), (4, 1))
+    y = torch.zeros(4, 64, dtype=torch.bfloat16, device="cuda")
+    ep.ep_combine(dev_bf16(out), torch.from_numpy(slot).cuda(), torch.from_numpy(w).cuda(), y, 4, 4)
+    got = inputs.bf16_bits_to_f32(host_bits(y))
+    assert (got == np.float32(c * 2.0 ** -23)).all()
+    np.testing.assert_array_equal(host_bits(y), oracle.combine_f32(out, slot, w))
+
+
 def test_capacity_overflow_is_skipped_and_flagged():
     cfg = inputs.CONFIGS["C1"]
     d = inputs.make_inputs(cfg)

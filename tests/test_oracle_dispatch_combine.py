@@ -82,6 +82,18 @@ def test_combine_order_of_k_matters_and_is_ascending():
     assert oracle.combine_f64(out, slot, w)[0, 0] == 2.0 ** -6     # the exact sum keeps it
 
 
+def test_combine_keeps_the_product_unrounded_inside_the_chain():
+    """A fused multiply-add rounds once: with acc = -c, w*v = c + c*2^-23 leaves c*2^-23 exactly,
+    whereas a rounded product (c + 2^-23) would leave 2^-23. c = 1 + 2^-7 is a bf16 number."""
+    c = 1.0078125
+    out = inputs.to_bf16_bits(np.array([[c], [c]], dtype=np.float32))
+    slot = np.array([[0, 1]], dtype=np.int32)
+    w = np.array([[-1.0, 1.0 + 2.0 ** -23]], dtype=np.float32)
+    y = inputs.bf16_bits_to_f32(oracle.combine_f32(out, slot, w))
+    assert y[0, 0] == np.float32(c * 2.0 ** -23) != np.float32(2.0 ** -23)
+    assert oracle.combine_f64(out, slot, w)[0, 0] == c * 2.0 ** -23
+
+
 def test_combine_single_rounding_of_the_product_matches_torch_cast():
     """K = 1: y = bf16(fp32(w * v)); numpy's fp32 multiply is the correctly rounded
     product and torch's CPU cast is the narrowing."""

@@ -75,6 +75,26 @@ def test_combine_partial_against_exact_rationals(seed):
         assert (np.abs(got[t] - y64[t]) <= _two_stage_bound(y64[t], rows)).all()
 
 
+def test_combine_partial_chain_runs_in_ascending_k_inside_a_rank():
+    """Three picks on one rank: big + small - big. Ascending k absorbs the small term (partial = 0);
+    any other order would keep it."""
+    out = inputs.to_bf16_bits(np.array([[2.0 ** 20], [2.0 ** -6], [2.0 ** 20]], dtype=np.float32))
+    pair_slot = np.array([[0, 1, 2]], dtype=np.int32)
+    recv_slot = np.zeros((1, 3), dtype=np.int32)
+    w = np.array([[1.0, 1.0, -1.0]], dtype=np.float32)
+    partial, y = oracle.combine_partial(out, pair_slot, recv_slot, w, 1)
+    assert inputs.bf16_bits_to_f32(partial)[0, 0] == 0.0 and inputs.bf16_bits_to_f32(y)[0, 0] == 0.0
+    w2 = np.array([[1.0, -1.0, 1.0]], dtype=np.float32)
+    pair_slot2 = np.array([[0, 2, 1]], dtype=np.int32)
+    partial, y = oracle.combine_partial(out, pair_slot2, recv_slot, w2, 1)
+    assert inputs.bf16_bits_to_f32(y)[0, 0] == 2.0 ** -6
+    # two ranks: the owner adds the partial rows in the order of their first k
+    recv_slot3 = np.array([[0, 1, 0]], dtype=np.int32)          # picks 0 and 2 on one rank, pick 1 on another
+    partial, y = oracle.combine_partial(out, pair_slot, recv_slot3, w, 2)
+    pf = inputs.bf16_bits_to_f32(partial)
+    assert pf[0, 0] == 0.0 and pf[1, 0] == 2.0 ** -6 and inputs.bf16_bits_to_f32(y)[0, 0] == 2.0 ** -6
+
+
 def test_combine_partial_closed_forms():
     # one rank: the partial row IS the one-stage result, and rounding it twice changes nothing
     cfg, idx, w, x, lay, out = _case(32, 64, 16, 4, 1, cid=82)
