@@ -12,12 +12,14 @@
 //   4. replays its tiles in (t,k) order with running counters that start at
 //      offset[bin] + earlier CTAs + earlier warps of this CTA.
 // Step 2 has three forms:
-//   single   one CTA holds every tile: nothing to exchange;
-//   cluster  up to 8 CTAs form one thread-block cluster and read each other's CTA
-//            totals through distributed shared memory between two cluster barriers:
-//            one launch, no global scratch (all five benchmark shapes take this path);
-//   global   larger batches: a first kernel writes cta_part[cta][bin] to the
-//            workspace; the main kernel, launched with programmatic stream
+//   single   one CTA of up to 32 warps holds every tile (up to 1024 tokens): nothing
+//            to exchange, one launch;
+//   cluster  up to 8 CTAs of 8 warps (up to 2048 tokens) form one thread-block cluster
+//            and read each other's CTA totals through distributed shared memory
+//            between two cluster barriers: one launch, no global scratch;
+//   global   larger batches, spread over up to 128 CTAs of 8 warps because the replay
+//            is throughput-bound per SM: a first kernel writes cta_part[cta][bin] to
+//            the workspace; the main kernel, launched with programmatic stream
 //            serialisation so that its histogram phase overlaps the first kernel,
 //            executes griddepcontrol.wait and then reads every cta_part row.
 // Bins: [0,E) experts, [E,E+R) rank hits, [E+R] ids outside [-1,E).
