@@ -118,6 +118,26 @@ def test_all_tokens_to_one_expert_and_all_masked():
     _full_path_check(cfg, -np.ones((T, K), np.int32), d["topk_weights"], d["x"])
 
 
+def test_layout_on_many_random_shapes():
+    """Seeded sweep over shapes that exercise the single-CTA, cluster and multi-CTA forms of the
+    layout, with masked and repeated ids mixed in; every integer output against the oracle."""
+    rng = np.random.default_rng(11)
+    for trial in range(48):
+        R = int(rng.choice([1, 2, 3, 4, 8, 16]))
+        E = R * int(rng.choice([1, 2, 5, 16, 32]))
+        K = int(rng.integers(1, min(8, E) + 1))
+        T = R * int(rng.integers(1, [40, 300, 1200][trial % 3]))
+        idx = rng.integers(0, E, size=(T, K)).astype(np.int32)
+        if trial % 4 == 1:
+            idx[rng.random((T, K)) < 0.15] = -1
+        if trial % 8 == 3:
+            idx[int(rng.integers(0, T)), int(rng.integers(0, K))] = E + 1
+        ref = oracle.layout(idx, E, R)
+        lay = _run_layout(idx, E, R)
+        assert_layout_equal(lay, ref)
+        assert ep.ep_status(lay.status) == ref.status, (trial, T, K, E, R)
+
+
 def test_empty_batch():
     E, R, K, H = 8, 2, 2, 64
     lay = ep.alloc_layout(0, K, E, R, fill=-7)
