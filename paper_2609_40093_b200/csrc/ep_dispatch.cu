@@ -60,23 +60,31 @@ dispatch_rows_kernel(const uint4 *__restrict__ x, const int32_t *__restrict__ re
     const int t = blockIdx.x * (blockDim.x / G) + threadIdx.x / G;
     if (t >= T) return;                                   // whole warps leave together (G % 32 == 0)
 
+    // the slot load and the first row loads are independent: issue both before anything waits on either
     int32_t slot = lane < K ? __ldg(recv_slot + (size_t)t * K + lane) : -1;
+    const uint4 *src = x + (size_t)t * vec_per_row;
+    uint4 buf[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const int v = g + u * G;
+        if (v < vec_per_row) buf[u] = ld_stream(src + v);
+    }
     if (slot >= capacity_rows) {
         flag_status(status, EP_STATUS_CAPACITY);
         slot = -1;
     }
     // the k's of a token that land on one rank share a slot: keep the lowest k
     const unsigned same = __match_any_sync(kFullMask, slot);
-    unsigned todo = __ballot_sync(kFullMask, slot >= 0 && (same & lanemask_lt()) == 0);
+    const unsigned todo = __ballot_sync(kFullMask, slot >= 0 && (same & lanemask_lt()) == 0);
 
-    const uint4 *src = x + (size_t)t * vec_per_row;
     for (int base = 0; base < vec_per_row; base += G * U) {  // trip count uniform over the warp
         const int v0 = base + g;
-        uint4 buf[U];
+        if (base > 0) {
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const int v = v0 + u * G;
-            if (v < vec_per_row) buf[u] = ld_stream(src + v);
+            for (int u = 0; u < U; ++u) {
+                const int v = v0 + u * G;
+                if (v < vec_per_row) buf[u] = ld_stream(src + v);
+            }
         }
         for (unsigned m = todo; m; m &= m - 1) {
             const int32_t row = __shfl_sync(kFullMask, slot, __ffs(m) - 1);
