@@ -5,7 +5,10 @@
 // columns (8 bf16). For a column it first issues the loads of up to kChunk rows
 // (they are independent: this is the memory-level parallelism), then folds them
 // into the eight accumulators strictly in k order. Slots and weights sit one per
-// lane and travel by warp shuffle. Small CTAs (128 threads, 63 registers, eight
+// lane and travel by warp shuffle. For K <= 8 the rows of a column are requested
+// in two halves and the next column's halves are requested between the two folds,
+// so that loads stay in flight during the arithmetic (measured -2 us of 166 at
+// T=8192, H=7168, K=8). Small CTAs (128 threads, 63 registers, eight
 // resident per SM) measured 5 % faster alone than 448-thread groups with two
 // columns per thread (165 vs 175 us at T=8192, H=7168, K=8).
 #include "ep_common.cuh"
@@ -15,6 +18,18 @@ namespace {
 
 constexpr int kBlock = 128;
 constexpr int kChunk = 8;   // rows in flight per column
+
+__device__ __forceinline__ void fma_row(float (&acc)[8], float w, const uint4 &r)
+{
+    acc[0] = __fmaf_rn(w, bf16_lo(r.x), acc[0]);
+    acc[1] = __fmaf_rn(w, bf16_hi(r.x), acc[1]);
+    acc[2] = __fmaf_rn(w, bf16_lo(r.y), acc[2]);
+    acc[3] = __fmaf_rn(w, bf16_hi(r.y), acc[3]);
+    acc[4] = __fmaf_rn(w, bf16_lo(r.z), acc[4]);
+    acc[5] = __fmaf_rn(w, bf16_hi(r.z), acc[5]);
+    acc[6] = __fmaf_rn(w, bf16_lo(r.w), acc[6]);
+    acc[7] = __fmaf_rn(w, bf16_hi(r.w), acc[7]);
+}
 
 template <int G>
 __global__ void __launch_bounds__(kBlock)
@@ -38,6 +53,64 @@ combine_rows_kernel(const uint4 *__restrict__ out, long long out_rows, const int
         }
     }
     uint4 *dst = y + (size_t)t * vec_per_row;
+    if (K <= kChunk) {
+        // K <= 8: the rows of a column are loaded in two halves, and the next column's halves are
+        // requested before the other half of this column is folded, so loads stay in flight during the
+        // arithmetic. The chain order (ascending k) is unchanged.
+        constexpr int kHalf = kChunk / 2;
+        const unsigned valid = __ballot_sync(kFullMask, my_slot >= 0);
+        uint4 lo[kHalf], hi[kHalf];
+        int v = g;
+        bool live = v < vec_per_row;
+#pragma unroll
+        for (int j = 0; j < kHalf; ++j) {
+            const int32_t s = __shfl_sync(kFullMask, my_slot, j);
+            if (live && ((valid >> j) & 1u)) lo[j] = ld_stream(out + (size_t)s * vec_per_row + v);
+        }
+#pragma unroll
+        for (int j = 0; j < kHalf; ++j) {
+            const int32_t s = __shfl_sync(kFullMask, my_slot, kHalf + j);
+            if (live && ((valid >> (kHalf + j)) & 1u)) hi[j] = ld_stream(out + (size_t)s * vec_per_row + v);
+        }
+        for (int base = 0; base < vec_per_row; base += G) {   // trip count uniform over the warp
+            const int vn = v + G;
+            const bool live_n = vn < vec_per_row;
+            float acc[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) acc[i] = 0.f;
+#pragma unroll
+            for (int j = 0; j < kHalf; ++j) {
+                const float w = __shfl_sync(kFullMask, my_w, j);
+                if (live && ((valid >> j) & 1u)) fma_row(acc, w, lo[j]);
+            }
+#pragma unroll
+            for (int j = 0; j < kHalf; ++j) {                 // low half of the next column
+                const int32_t s = __shfl_sync(kFullMask, my_slot, j);
+                if (live_n && ((valid >> j) & 1u)) lo[j] = ld_stream(out + (size_t)s * vec_per_row + vn);
+            }
+#pragma unroll
+            for (int j = 0; j < kHalf; ++j) {
+                const float w = __shfl_sync(kFullMask, my_w, kHalf + j);
+                if (live && ((valid >> (kHalf + j)) & 1u)) fma_row(acc, w, hi[j]);
+            }
+#pragma unroll
+            for (int j = 0; j < kHalf; ++j) {                 // high half of the next column
+                const int32_t s = __shfl_sync(kFullMask, my_slot, kHalf + j);
+                if (live_n && ((valid >> (kHalf + j)) & 1u)) hi[j] = ld_stream(out + (size_t)s * vec_per_row + vn);
+            }
+            if (live) {
+                uint4 o;
+                o.x = pack_bf16x2(acc[0], acc[1]);
+                o.y = pack_bf16x2(acc[2], acc[3]);
+                o.z = pack_bf16x2(acc[4], acc[5]);
+                o.w = pack_bf16x2(acc[6], acc[7]);
+                st_stream(dst + v, o);
+            }
+            v = vn;
+            live = live_n;
+        }
+        return;
+    }
     for (int base = 0; base < vec_per_row; base += G) {   // trip count uniform over the warp
         const int v = base + g;
         const bool live = v < vec_per_row;
