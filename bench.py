@@ -31,7 +31,7 @@ NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes per launch of the dominant kernel from the committed ncu capture
 # (profiles/): filled in per workload once measured, else null.
-NCU_TRAFFIC_BYTES = {("C4", "combine_rows_kernel"): 1037.9e6, ("C4", "dispatch_rows_kernel"): 681.6e6}
+NCU_TRAFFIC_BYTES = {("C4", "combine_rows_kernel"): 1038.7e6, ("C4", "dispatch_rows_kernel"): 680.8e6}
 L2_BYTES = 126e6
 
 
