@@ -28,6 +28,8 @@ EDGE = [  # T, H, E, K, R, routing
     (1088, 64, 4096, 32, 64, "uniform"),   # every maximum at once: K=32, E=4096, R=64
     (40000, 8, 16, 2, 8, "uniform"),       # more than 1024*32 tokens: layout tiles of 64 tokens, 16-byte rows
     (33 * 8, 40, 24, 5, 8, "zipf_identity"),
+    (65536, 8, 256, 8, 8, "burst"),        # 128 layout CTAs, tiles of 64 tokens, half a million pairs
+    (2048, 24, 128, 6, 8, "zipf"),         # the largest batch that takes the one-cluster layout
 ]
 
 
