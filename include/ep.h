@@ -104,6 +104,25 @@ int ep_layout(const ep_shape_t *shape, const int32_t *topk_idx, const ep_layout_
               void *workspace, size_t workspace_bytes, void *stream);
 
 /*
+ * The two halves of ep_layout as separate calls, so that they can run on
+ * different streams: dispatch needs only the receive-row half, combine only the
+ * pair half, and the pair half can therefore be computed while dispatch moves
+ * rows (Section 4.5 blames the routing-metadata step for the cost of
+ * routing-aware transfers; this takes most of it off the critical path).
+ *   ep_layout_ranks  writes rank_rows, rank_row_offsets, src_row_offsets,
+ *                    recv_slot, recv_token and status;
+ *   ep_layout_pairs  writes expert_counts, expert_offsets, pair_slot, pair_row
+ *                    and pair_token, and never touches status.
+ * Each reads only topk_idx; the fields of `out` a call does not write may be
+ * NULL. Together they produce exactly what ep_layout produces. Calls that may
+ * overlap need workspaces of their own (ep_layout_workspace_bytes each).
+ */
+int ep_layout_ranks(const ep_shape_t *shape, const int32_t *topk_idx, const ep_layout_t *out,
+                    void *workspace, size_t workspace_bytes, void *stream);
+int ep_layout_pairs(const ep_shape_t *shape, const int32_t *topk_idx, const ep_layout_t *out,
+                    void *workspace, size_t workspace_bytes, void *stream);
+
+/*
  * Layout without any allocation (the paper has no counterpart; this entry point
  * exists for integration reasons only). Some callers cannot obtain device
  * memory at the point where they need a layout: code running inside a serving

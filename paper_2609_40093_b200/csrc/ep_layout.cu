@@ -41,6 +41,7 @@ constexpr int kMaxCtasGlobal = 128;
 constexpr size_t kSmemBudget = 200 * 1024;
 
 enum { kModeSingle = 0, kModeCluster = 1, kModeGlobal = 2 };
+enum { kPartRanks = 1, kPartPairs = 2 };
 
 struct LayoutPlan {
     int mode;
@@ -122,6 +123,8 @@ struct LayoutArgs {
     int T, K, E, R, Tr;
     FastDiv by_El, by_K, by_Tr;
     int tile_tokens, n_tiles, bins, n_ctas, mode;
+    int parts;   // kPartRanks | kPartPairs: which outputs this call writes
+    int blo;     // first bin in use: 0, or E when only the receive-row half is wanted
 };
 
 // The warp copies the expert ids of the 32 tokens [tb, tb+32) into ids[32*K] (coalesced, all loads in
@@ -152,7 +155,7 @@ template <bool kShared>
 __device__ __forceinline__ void count_tile(const LayoutArgs &a, int32_t *hist, int32_t *ids, int tile, int lane)
 {
     if (!kShared) {
-        for (int b = lane; b < a.bins; b += 32) hist[b] = 0;
+        for (int b = a.blo + lane; b < a.bins; b += 32) hist[b] = 0;
         __syncwarp();
     }
     if (tile >= a.n_tiles) return;
@@ -163,8 +166,11 @@ __device__ __forceinline__ void count_tile(const LayoutArgs &a, int32_t *hist, i
         const int n_items = stage_group(a, ids, tb, t1, lane);
         for (int i = lane; i < n_items; i += 32) {                   // experts: any order
             const int e = ids[i];
-            if (e >= 0 && e < a.E) atomicAdd(hist + e, 1);
-            else if (e != -1) ++bad;
+            if (e >= 0 && e < a.E) {
+                if (a.blo == 0) atomicAdd(hist + e, 1);
+            } else if (e != -1) {
+                ++bad;
+            }
         }
         const unsigned long long mask = token_rank_mask(a, ids, lane);   // rank hits: token per lane, ballot per rank
         for (int r = 0; r < a.R; ++r) {
@@ -222,12 +228,12 @@ __global__ void __launch_bounds__(kMaxWarps * 32) layout_cta_count_kernel(Layout
     extern __shared__ int32_t smem[];
     const int warps = blockDim.x >> 5, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     // one histogram for the CTA (first `bins` words), per-warp id staging behind it
-    for (int b = threadIdx.x; b < a.bins; b += blockDim.x) smem[b] = 0;
+    for (int b = a.blo + threadIdx.x; b < a.bins; b += blockDim.x) smem[b] = 0;
     __syncthreads();
     count_tile<true>(a, smem, smem + a.bins + warp * 32 * a.K, blockIdx.x * warps + warp, lane);
     __syncthreads();
     int32_t *dst = a.cta_part + (size_t)blockIdx.x * a.bins;
-    for (int b = threadIdx.x; b < a.bins; b += blockDim.x) dst[b] = smem[b];
+    for (int b = a.blo + threadIdx.x; b < a.bins; b += blockDim.x) dst[b] = smem[b];
 }
 
 // ---------------------------------------------------------------- main kernel
@@ -252,7 +258,8 @@ __global__ void __launch_bounds__(kMaxWarpsSingle * 32) layout_assign_kernel(Lay
     count_tile<false>(a, run, ids, tile, lane);
     __syncthreads();
     EP_STAMP(1);
-    for (int b = threadIdx.x; b < a.bins; b += blockDim.x) {         // this CTA's total per bin
+    const bool ranks = a.parts & kPartRanks, pairs = a.parts & kPartPairs;
+    for (int b = a.blo + threadIdx.x; b < a.bins; b += blockDim.x) {  // this CTA's total per bin
         int32_t mine = 0;
         for (int w = 0; w < warps; ++w) mine += smem[w * pw + b];
         cta_tot[b] = mine;
@@ -261,7 +268,7 @@ __global__ void __launch_bounds__(kMaxWarpsSingle * 32) layout_assign_kernel(Lay
     else if (a.mode == kModeGlobal) pdl_wait();                      // cta_part is complete and visible
     EP_STAMP(2);
     // per bin: count in earlier CTAs and grand total (each thread reads the cta_tot entries it wrote itself)
-    for (int b = threadIdx.x; b < a.bins; b += blockDim.x) {
+    for (int b = a.blo + threadIdx.x; b < a.bins; b += blockDim.x) {
         int32_t before = 0, total = 0;
         if (a.mode == kModeCluster) {
             cg::cluster_group cluster = cg::this_cluster();
@@ -284,7 +291,8 @@ __global__ void __launch_bounds__(kMaxWarpsSingle * 32) layout_assign_kernel(Lay
         pre[b] = before;
         if (b < nb) tot[b] = total;
         if (blockIdx.x == 0) {
-            if (b < a.E) a.out.expert_counts[b] = total;
+            if (b < a.E) a.out.expert_counts[b] = total;               // only reached when the pair half is wanted
+            else if (!ranks) continue;
             else if (b < nb) a.out.rank_rows[b - a.E] = total;
             else *a.out.status = total ? EP_STATUS_BAD_INDEX : 0;
         }
@@ -293,16 +301,19 @@ __global__ void __launch_bounds__(kMaxWarpsSingle * 32) layout_assign_kernel(Lay
     else __syncthreads();
     EP_STAMP(3);
     // one exclusive scan over [experts | ranks]: S[e] = expert offset, S[E + r] - S[E] = rank row offset
-    block_exclusive_scan_smem(tot, nb, sh);
-    const int32_t n_pairs = tot[a.E];
+    block_exclusive_scan_smem(tot + a.blo, nb - a.blo, sh);
+    const int32_t n_pairs = tot[a.E];                                // 0 when the scan started at the rank bins
     if (blockIdx.x == 0) {
-        for (int e = threadIdx.x; e <= a.E; e += blockDim.x) a.out.expert_offsets[e] = tot[e];
-        for (int r = threadIdx.x; r <= a.R; r += blockDim.x) a.out.rank_row_offsets[r] = tot[a.E + r] - n_pairs;
-        for (int r = threadIdx.x; r < a.R; r += blockDim.x)
-            a.out.src_row_offsets[r * (a.R + 1) + a.R] = tot[a.E + r + 1] - n_pairs;
+        if (pairs)
+            for (int e = threadIdx.x; e <= a.E; e += blockDim.x) a.out.expert_offsets[e] = tot[e];
+        if (ranks) {
+            for (int r = threadIdx.x; r <= a.R; r += blockDim.x) a.out.rank_row_offsets[r] = tot[a.E + r] - n_pairs;
+            for (int r = threadIdx.x; r < a.R; r += blockDim.x)
+                a.out.src_row_offsets[r * (a.R + 1) + a.R] = tot[a.E + r + 1] - n_pairs;
+        }
     }
     // next free slot of every bin for every warp: offset + earlier CTAs + earlier warps of this CTA
-    for (int b = threadIdx.x; b < nb; b += blockDim.x) {
+    for (int b = a.blo + threadIdx.x; b < nb; b += blockDim.x) {
         int32_t running = pre[b] + (b < a.E ? tot[b] : tot[b] - n_pairs);
         for (int w = 0; w < warps; ++w) {
             const int32_t v = smem[w * pw + b];
@@ -331,7 +342,7 @@ __global__ void __launch_bounds__(kMaxWarpsSingle * 32) layout_assign_kernel(Lay
         __syncwarp();
         if (live) {
             const int s = fdiv(t, a.by_Tr);
-            if (t == s * a.Tr)                       // first token of source rank s
+            if (ranks && t == s * a.Tr)              // first token of source rank s
                 for (int r = 0; r < a.R; ++r)
                     a.out.src_row_offsets[r * (a.R + 1) + s] = run[a.E + r] + __popc(bal[r] & lt);
             unsigned long long seen = 0ull;
@@ -341,7 +352,7 @@ __global__ void __launch_bounds__(kMaxWarpsSingle * 32) layout_assign_kernel(Lay
                 if (e >= 0 && e < a.E) {
                     const int r = fdiv(e, a.by_El);
                     row = run[a.E + r] + __popc(bal[r] & lt);
-                    if (!((seen >> r) & 1ull)) {
+                    if (ranks && !((seen >> r) & 1ull)) {
                         a.out.recv_token[row] = t;
                         seen |= 1ull << r;
                     }
@@ -352,9 +363,14 @@ __global__ void __launch_bounds__(kMaxWarpsSingle * 32) layout_assign_kernel(Lay
         __syncwarp();
         for (int r = lane; r < a.R; r += 32) run[a.E + r] += __popc(bal[r]);
         __syncwarp();
+        int32_t *recv_slot = a.out.recv_slot + (size_t)tb * a.K;
+        if (!pairs) {                                // receive-row half only: publish the rows and go on
+            for (int i = lane; i < n_items; i += 32) recv_slot[i] = slot_s[i];
+            __syncwarp();
+            continue;
+        }
         // --- pair slots: the items of these tokens, 32 at a time in (t,k) order
         int32_t *pair_slot = a.out.pair_slot + (size_t)tb * a.K;
-        int32_t *recv_slot = a.out.recv_slot + (size_t)tb * a.K;
         for (int j = 0; j < n_items; j += 32) {
             const int i = j + lane;
             const bool act = i < n_items;
@@ -367,12 +383,12 @@ __global__ void __launch_bounds__(kMaxWarpsSingle * 32) layout_assign_kernel(Lay
                 const int32_t p = first + __popc(m & lt);
                 const int32_t row = slot_s[i];
                 pair_slot[i] = p;
-                recv_slot[i] = row;
+                if (ranks) recv_slot[i] = row;
                 a.out.pair_token[p] = tb + fdiv(i, a.by_K);
                 a.out.pair_row[p] = row;
             } else if (act) {
                 pair_slot[i] = -1;
-                recv_slot[i] = -1;
+                if (ranks) recv_slot[i] = -1;
             }
             __syncwarp();
             if (valid && (m >> lane) <= 1u) run[e] = first + __popc(m);   // highest lane of the group
@@ -395,31 +411,36 @@ extern "C" size_t ep_layout_workspace_bytes(const ep_shape_t *shape)
     return ep::make_plan(*shape).workspace_bytes;
 }
 
-extern "C" int ep_layout(const ep_shape_t *shape, const int32_t *topk_idx, const ep_layout_t *out,
-                         void *workspace, size_t workspace_bytes, void *stream_)
+namespace ep {
+namespace {
+
+int run_layout(const ep_shape_t *shape, const int32_t *topk_idx, const ep_layout_t *out, void *workspace,
+               size_t workspace_bytes, void *stream_, int parts)
 {
-    using namespace ep;
     int rc = check_shape(shape, false);
     if (rc != EP_OK) return rc;
     if (!out || !workspace) return EP_ERR_NULL;
-    if (!out->expert_counts || !out->expert_offsets || !out->rank_rows || !out->rank_row_offsets ||
-        !out->src_row_offsets || !out->status)
-        return EP_ERR_NULL;
-    if (shape->num_tokens > 0 && (!out->recv_slot || !out->pair_slot || !out->recv_token || !out->pair_row ||
-                                  !out->pair_token))
-        return EP_ERR_NULL;
+    const bool ranks = parts & kPartRanks, pairs = parts & kPartPairs;
+    if (ranks && (!out->rank_rows || !out->rank_row_offsets || !out->src_row_offsets || !out->status)) return EP_ERR_NULL;
+    if (pairs && (!out->expert_counts || !out->expert_offsets)) return EP_ERR_NULL;
+    if (shape->num_tokens > 0 && ranks && (!out->recv_slot || !out->recv_token)) return EP_ERR_NULL;
+    if (shape->num_tokens > 0 && pairs && (!out->pair_slot || !out->pair_row || !out->pair_token)) return EP_ERR_NULL;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
     const LayoutPlan plan = make_plan(*shape);
     if (workspace_bytes < plan.workspace_bytes) return EP_ERR_CAPACITY;
     if (!aligned16(workspace)) return EP_ERR_INVALID_ARG;
     const int T = shape->num_tokens, E = shape->num_experts, R = shape->num_ranks;
     if (T == 0) {
-        EP_CUDA_TRY(cudaMemsetAsync(out->expert_counts, 0, sizeof(int32_t) * E, stream));
-        EP_CUDA_TRY(cudaMemsetAsync(out->expert_offsets, 0, sizeof(int32_t) * (E + 1), stream));
-        EP_CUDA_TRY(cudaMemsetAsync(out->rank_rows, 0, sizeof(int32_t) * R, stream));
-        EP_CUDA_TRY(cudaMemsetAsync(out->rank_row_offsets, 0, sizeof(int32_t) * (R + 1), stream));
-        EP_CUDA_TRY(cudaMemsetAsync(out->src_row_offsets, 0, sizeof(int32_t) * R * (R + 1), stream));
-        EP_CUDA_TRY(cudaMemsetAsync(out->status, 0, sizeof(int32_t), stream));
+        if (pairs) {
+            EP_CUDA_TRY(cudaMemsetAsync(out->expert_counts, 0, sizeof(int32_t) * E, stream));
+            EP_CUDA_TRY(cudaMemsetAsync(out->expert_offsets, 0, sizeof(int32_t) * (E + 1), stream));
+        }
+        if (ranks) {
+            EP_CUDA_TRY(cudaMemsetAsync(out->rank_rows, 0, sizeof(int32_t) * R, stream));
+            EP_CUDA_TRY(cudaMemsetAsync(out->rank_row_offsets, 0, sizeof(int32_t) * (R + 1), stream));
+            EP_CUDA_TRY(cudaMemsetAsync(out->src_row_offsets, 0, sizeof(int32_t) * R * (R + 1), stream));
+            EP_CUDA_TRY(cudaMemsetAsync(out->status, 0, sizeof(int32_t), stream));
+        }
         return EP_OK;
     }
     if (!topk_idx) return EP_ERR_NULL;
@@ -432,6 +453,8 @@ extern "C" int ep_layout(const ep_shape_t *shape, const int32_t *topk_idx, const
     a.by_El = make_fastdiv(E / R); a.by_K = make_fastdiv(shape->top_k); a.by_Tr = make_fastdiv(T / R);
     a.tile_tokens = plan.tile_tokens; a.n_tiles = plan.n_tiles; a.bins = plan.bins; a.n_ctas = plan.n_ctas;
     a.mode = plan.mode;
+    a.parts = parts;
+    a.blo = pairs ? 0 : E;
 #ifdef EP_LAYOUT_TIMING
     a.dbg = g_timing_buf;
 #endif
@@ -470,6 +493,27 @@ extern "C" int ep_layout(const ep_shape_t *shape, const int32_t *topk_idx, const
     EP_CUDA_TRY(cudaLaunchKernelEx(&cfg, layout_assign_kernel, a));
     EP_LAUNCH_CHECK(launched);
     return EP_OK;
+}
+
+}  // namespace
+}  // namespace ep
+
+extern "C" int ep_layout(const ep_shape_t *shape, const int32_t *topk_idx, const ep_layout_t *out,
+                         void *workspace, size_t workspace_bytes, void *stream)
+{
+    return ep::run_layout(shape, topk_idx, out, workspace, workspace_bytes, stream, ep::kPartRanks | ep::kPartPairs);
+}
+
+extern "C" int ep_layout_ranks(const ep_shape_t *shape, const int32_t *topk_idx, const ep_layout_t *out,
+                               void *workspace, size_t workspace_bytes, void *stream)
+{
+    return ep::run_layout(shape, topk_idx, out, workspace, workspace_bytes, stream, ep::kPartRanks);
+}
+
+extern "C" int ep_layout_pairs(const ep_shape_t *shape, const int32_t *topk_idx, const ep_layout_t *out,
+                               void *workspace, size_t workspace_bytes, void *stream)
+{
+    return ep::run_layout(shape, topk_idx, out, workspace, workspace_bytes, stream, ep::kPartPairs);
 }
 
 // ---------------------------------------------------------------------------

@@ -22,7 +22,7 @@ STATUS_TIMEOUT = 4
 PROBE_READ, PROBE_WRITE, PROBE_COPY, PROBE_MEMCPY = 0, 1, 2, 3
 
 EXPORTS = [
-    "ep_layout_workspace_bytes", "ep_layout", "ep_layout_static", "ep_layout_static_scratch_bytes", "ep_dispatch", "ep_combine", "ep_group",
+    "ep_layout_workspace_bytes", "ep_layout", "ep_layout_ranks", "ep_layout_pairs", "ep_layout_static", "ep_layout_static_scratch_bytes", "ep_dispatch", "ep_combine", "ep_group",
     "ep_combine_partial", "ep_dense_allgather", "ep_dense_reduce_scatter",
     "ep_host_roundtrip", "ep_wait_senders", "ep_post_flags", "ep_host_step_pipelined",
     "ep_dispatch_copy_engine", "ep_host_step_arena_bytes", "ep_host_step", "ep_status",
@@ -63,6 +63,10 @@ def lib() -> ctypes.CDLL:
         L.ep_layout_workspace_bytes.restype = sz
         L.ep_layout_workspace_bytes.argtypes = [sp]
         L.ep_layout.argtypes = [sp, vp, ctypes.POINTER(_Layout), vp, sz, vp]
+        L.ep_layout_ranks.argtypes = [sp, vp, ctypes.POINTER(_Layout), vp, sz, vp]
+        L.ep_layout_pairs.argtypes = [sp, vp, ctypes.POINTER(_Layout), vp, sz, vp]
+        L.ep_layout_ranks.restype = i32
+        L.ep_layout_pairs.restype = i32
         L.ep_layout_static.argtypes = [sp, vp, ctypes.POINTER(_Layout), vp]
         L.ep_layout_static.restype = i32
         L.ep_layout_static_scratch_bytes.restype = sz
@@ -159,6 +163,25 @@ def ep_layout(topk_idx: torch.Tensor, E: int, R: int, out: Layout = None, worksp
     _check(lib().ep_layout(ctypes.byref(_shape(T, K, 8, E, R)), _ptr(topk_idx), ctypes.byref(st), _ptr(workspace),
                            workspace.numel(), _stream()), "ep_layout")
     return out
+
+
+def _layout_half(fn_name, topk_idx, E, R, out, workspace, stream):
+    T, K = topk_idx.shape
+    st = out.as_struct()
+    sp = ctypes.c_void_p(stream.cuda_stream) if stream is not None else _stream()
+    _check(getattr(lib(), fn_name)(ctypes.byref(_shape(T, K, 8, E, R)), _ptr(topk_idx), ctypes.byref(st), _ptr(workspace),
+                                   workspace.numel(), sp), fn_name)
+    return out
+
+
+def ep_layout_ranks(topk_idx, E, R, out: Layout, workspace, stream=None) -> Layout:
+    """The receive-row half of `ep_layout` (what dispatch needs)."""
+    return _layout_half("ep_layout_ranks", topk_idx, E, R, out, workspace, stream)
+
+
+def ep_layout_pairs(topk_idx, E, R, out: Layout, workspace, stream=None) -> Layout:
+    """The pair-space half of `ep_layout` (what grouping and combine need); may run on another stream."""
+    return _layout_half("ep_layout_pairs", topk_idx, E, R, out, workspace, stream)
 
 
 def ep_layout_static(topk_idx: torch.Tensor, E: int, R: int, out: Layout) -> Layout:

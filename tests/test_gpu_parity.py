@@ -140,6 +140,28 @@ def test_layout_on_many_random_shapes():
         assert ep.ep_status(lay.status) == ref.status, (trial, T, K, E, R)
 
 
+@pytest.mark.parametrize("name", ["C1", "C3", "C4"])
+def test_layout_halves_on_two_streams_equal_the_whole(name):
+    """ep_layout_ranks and ep_layout_pairs, each on its own stream with its own workspace, fill
+    disjoint fields; together they must give what ep_layout gives (and the oracle)."""
+    cfg = inputs.CONFIGS[name]
+    idx = inputs.make_topk_idx(cfg)
+    idx[5 % cfg.T, 0] = -1
+    ref = oracle.layout(idx, cfg.E, cfg.R)
+    idx_d = torch.from_numpy(idx).cuda()
+    lay = ep.alloc_layout(cfg.T, cfg.K, cfg.E, cfg.R, fill=-7)
+    nbytes = max(16, ep.ep_layout_workspace_bytes(cfg.T, cfg.K, cfg.E, cfg.R))
+    ws1, ws2 = (torch.empty(nbytes, dtype=torch.uint8, device="cuda") for _ in range(2))
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    for _ in range(3):
+        ep.ep_layout_pairs(idx_d, cfg.E, cfg.R, lay, ws2, stream=s2)
+        ep.ep_layout_ranks(idx_d, cfg.E, cfg.R, lay, ws1, stream=s1)
+    torch.cuda.synchronize()
+    assert_layout_equal(lay, ref)
+    assert ep.ep_status(lay.status) == ref.status
+
+
 def test_empty_batch():
     E, R, K, H = 8, 2, 2, 64
     lay = ep.alloc_layout(0, K, E, R, fill=-7)
