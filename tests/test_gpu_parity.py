@@ -30,6 +30,8 @@ EDGE = [  # T, H, E, K, R, routing
     (33 * 8, 40, 24, 5, 8, "zipf_identity"),
     (65536, 8, 256, 8, 8, "burst"),        # 128 layout CTAs, tiles of 64 tokens, half a million pairs
     (2048, 24, 128, 6, 8, "zipf"),         # the largest batch that takes the one-cluster layout
+    (16, 16384, 8, 2, 4, "uniform"),       # rows longer than one pass of the widest thread group
+    (64, 8200, 64, 20, 4, "uniform"),      # K > 8: combine's chunked path; 1025 vectors per row
 ]
 
 
@@ -108,6 +110,17 @@ def test_masked_duplicate_and_bad_ids():
     idx[200, 0] = -9
     lay, ref = _full_path_check(cfg, idx, d["topk_weights"], d["x"])
     assert ref.status == ep.STATUS_BAD_INDEX
+
+
+def test_wide_top_k_with_masks():
+    rng = np.random.default_rng(9)
+    T, H, E, K, R = 96, 264, 96, 32, 8
+    cfg = inputs.custom_config(T, H, E, K, R, config_id=63)
+    d = inputs.make_inputs(cfg)
+    idx = d["topk_idx"].copy()
+    idx[rng.random((T, K)) < 0.3] = -1
+    idx[0, :] = -1
+    _full_path_check(cfg, idx, d["topk_weights"], d["x"])
 
 
 def test_all_tokens_to_one_expert_and_all_masked():
