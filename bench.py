@@ -51,7 +51,7 @@ class L2Flush:
         torch.sum(self.r)
 
 
-def LAUNCHES_PER_STEP(ep, step):
+def launches_per_step(ep, step):
     """Kernels one direct (non-graph) step launches, counted by the library."""
     n0 = ep.ep_launch_count()
     step()
@@ -469,7 +469,7 @@ def main():
         rep.barrier()
         launches = ep.ep_launch_count() - launches0
         if graph is not None:                   # replays launch the captured kernels without passing through the library
-            launches = args.steps * LAUNCHES_PER_STEP(ep, step)
+            launches = args.steps * launches_per_step(ep, step)
         total_ms = rep.max_over_ranks(sum(s.elapsed_time(e) for s, e in zip(s_ev, e_ev)))
         # per-kernel figures from a separate pass of direct launches, each step after a flush
         evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(min(args.steps, 50))]

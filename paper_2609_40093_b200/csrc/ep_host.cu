@@ -294,7 +294,12 @@ extern "C" int ep_probe_bandwidth(int kind, void *dst, const void *src, size_t b
     EP_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
     cudaEvent_t e0, e1;
     EP_CUDA_TRY(cudaEventCreate(&e0));
-    EP_CUDA_TRY(cudaEventCreate(&e1));
+    cudaError_t ce = cudaEventCreate(&e1);
+    if (ce != cudaSuccess) {
+        cudaEventDestroy(e0);
+        note_cuda_error(ce);
+        return EP_ERR_CUDA;
+    }
     const size_t n_vec = bytes / 16;
     const int block = 256, grid = sms * 8;
     float best_ms = 1e30f;

@@ -25,6 +25,7 @@
 // Bins: [0,E) experts, [E,E+R) rank hits, [E+R] ids outside [-1,E).
 #include <cooperative_groups.h>
 
+#include <atomic>
 #include <mutex>
 
 #include "ep_common.cuh"
@@ -459,13 +460,14 @@ int run_layout(const ep_shape_t *shape, const int32_t *topk_idx, const ep_layout
     a.dbg = g_timing_buf;
 #endif
 
-    static bool attr_done[64] = {};
+    static std::atomic<bool> attr_done[64] = {};       // per device: dynamic shared memory limit raised
     int dev = 0;
     EP_CUDA_TRY(cudaGetDevice(&dev));
-    if (dev < 64 && !attr_done[dev]) {
+    if (dev < 0 || dev >= 64) return EP_ERR_INVALID_ARG;
+    if (!attr_done[dev].load(std::memory_order_acquire)) {
         EP_CUDA_TRY(cudaFuncSetAttribute(layout_cta_count_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget));
         EP_CUDA_TRY(cudaFuncSetAttribute(layout_assign_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget));
-        attr_done[dev] = true;
+        attr_done[dev].store(true, std::memory_order_release);
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(plan.n_ctas);
