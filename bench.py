@@ -401,10 +401,10 @@ def main():
             ep.ep_layout(idx, E, R, out=lay, workspace=ws)
         else:
             fork_ev.record(main)                      # the side stream starts after everything queued so far
+            ep.ep_layout_ranks(idx, E, R, lay, ws)    # critical path first
             side.wait_event(fork_ev)
             ep.ep_layout_pairs(idx, E, R, lay, ws2, stream=side)
             join_ev.record(side)
-            ep.ep_layout_ranks(idx, E, R, lay, ws)
         if events:
             events[1].record()
         ep.ep_dispatch(x, lay.recv_slot, recv, E, R, status=lay.status)
