@@ -104,7 +104,17 @@ def _shape(T, K, H, E, R) -> _Shape:
 
 
 def _ptr(t):
-    return None if t is None else ctypes.c_void_p(t.data_ptr())
+    """Address of a tensor's first element; the library sees dense row-major memory only."""
+    if t is None:
+        return None
+    if not t.is_contiguous():
+        raise ValueError("the EP library needs contiguous tensors")
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _want(t, dtype, name):
+    if t.dtype != dtype:
+        raise TypeError(f"{name} must be {dtype}, got {t.dtype}")
 
 
 def _stream():
@@ -154,6 +164,7 @@ def ep_layout_workspace_bytes(T, K, E, R) -> int:
 
 
 def ep_layout(topk_idx: torch.Tensor, E: int, R: int, out: Layout = None, workspace: torch.Tensor = None) -> Layout:
+    _want(topk_idx, torch.int32, "topk_idx")
     T, K = topk_idx.shape
     if out is None:
         out = alloc_layout(T, K, E, R, device=topk_idx.device)
@@ -200,6 +211,7 @@ def ep_layout_static_scratch_bytes() -> int:
 
 
 def ep_dispatch(x: torch.Tensor, recv_slot: torch.Tensor, recv: torch.Tensor, E: int, R: int, status=None):
+    _want(x, torch.bfloat16, "x"), _want(recv, torch.bfloat16, "recv"), _want(recv_slot, torch.int32, "recv_slot")
     T, H = x.shape
     K = recv_slot.shape[1]
     _check(lib().ep_dispatch(ctypes.byref(_shape(T, K, H, E, R)), _ptr(x), _ptr(recv_slot), _ptr(recv),
@@ -209,6 +221,8 @@ def ep_dispatch(x: torch.Tensor, recv_slot: torch.Tensor, recv: torch.Tensor, E:
 
 def ep_combine(out: torch.Tensor, slot: torch.Tensor, topk_weights: torch.Tensor, y: torch.Tensor, E: int, R: int,
                status=None):
+    _want(out, torch.bfloat16, "out"), _want(y, torch.bfloat16, "y"), _want(slot, torch.int32, "slot")
+    _want(topk_weights, torch.float32, "topk_weights")
     T, K = slot.shape
     H = out.shape[1]
     _check(lib().ep_combine(ctypes.byref(_shape(T, K, H, E, R)), _ptr(out), out.shape[0], _ptr(slot),

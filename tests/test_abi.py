@@ -58,6 +58,19 @@ def test_host_side_validation_needs_no_gpu():
     assert L.ep_launch_count() == 0 or L.ep_launch_count() > 0
 
 
+def test_binding_rejects_wrong_dtypes_and_strided_tensors():
+    import torch
+    x = torch.zeros(4, 16, dtype=torch.float32)
+    slot = torch.zeros(4, 2, dtype=torch.int32)
+    with pytest.raises(TypeError, match="bfloat16"):
+        ep.ep_dispatch(x, slot, x, 4, 2)
+    xb = torch.zeros(4, 32, dtype=torch.bfloat16)[:, ::2]
+    with pytest.raises(ValueError, match="contiguous"):
+        ep.ep_dispatch(xb, slot, torch.zeros(8, 16, dtype=torch.bfloat16), 4, 2)
+    with pytest.raises(TypeError, match="int32"):
+        ep.ep_layout(torch.zeros(4, 2, dtype=torch.int64), 4, 2)
+
+
 def test_binding_refuses_to_run_without_the_library(monkeypatch, tmp_path):
     monkeypatch.setattr(ep, "_lib", None)
     monkeypatch.setattr(ep, "_LIB_PATH", str(tmp_path / "absent.so"))
