@@ -175,6 +175,47 @@ def test_layout_halves_on_two_streams_equal_the_whole(name):
     assert ep.ep_status(lay.status) == ref.status
 
 
+def test_whole_step_replays_from_a_cuda_graph():
+    """No call of the path synchronises or allocates, so one step can be captured once and replayed
+    on new routing tables and activations written into the same buffers."""
+    cfg = inputs.CONFIGS["C3"]
+    T, K, H, E, R = cfg.T, cfg.K, cfg.H, cfg.E, cfg.R
+    idx_d = torch.zeros(T, K, dtype=torch.int32, device="cuda")
+    w_d = torch.zeros(T, K, dtype=torch.float32, device="cuda")
+    x_d = torch.zeros(T, H, dtype=torch.bfloat16, device="cuda")
+    lay = ep.alloc_layout(T, K, E, R)
+    ws = torch.empty(max(16, ep.ep_layout_workspace_bytes(T, K, E, R)), dtype=torch.uint8, device="cuda")
+    recv = torch.zeros(T * min(K, R), H, dtype=torch.bfloat16, device="cuda")
+    grouped = torch.zeros(T * K, H, dtype=torch.bfloat16, device="cuda")
+    y = torch.zeros(T, H, dtype=torch.bfloat16, device="cuda")
+
+    def step():
+        ep.ep_layout(idx_d, E, R, out=lay, workspace=ws)
+        ep.ep_dispatch(x_d, lay.recv_slot, recv, E, R, status=lay.status)
+        ep.ep_group(recv, lay, grouped, E, R, status=lay.status)
+        ep.ep_combine(grouped, lay.pair_slot, w_d, y, E, R, status=lay.status)
+
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):                       # first calls (per-device set-up) outside the capture
+        step()
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        step()
+    for seed in (3, 4):
+        d = inputs.make_inputs(cfg, seed)
+        idx_d.copy_(torch.from_numpy(d["topk_idx"]))
+        w_d.copy_(torch.from_numpy(d["topk_weights"]))
+        x_d.copy_(dev_bf16(d["x"]))
+        graph.replay()
+        torch.cuda.synchronize()
+        ref = oracle.layout(d["topk_idx"], E, R)
+        want = oracle.combine_f32(oracle.dispatch(d["x"], ref.recv_slot, ref.n_recv)[ref.pair_row], ref.pair_slot,
+                                  d["topk_weights"])
+        np.testing.assert_array_equal(host_bits(y), want)
+        assert ep.ep_status(lay.status) == 0
+
+
 def test_empty_batch():
     E, R, K, H = 8, 2, 2, 64
     lay = ep.alloc_layout(0, K, E, R, fill=-7)
