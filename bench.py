@@ -521,6 +521,17 @@ def main():
     d2h = y_h.numel() * 2 + 4
     del arena
 
+    # the library's own stream probes on this GPU, beside the measured copy peak
+    probes = None
+    if not cfg.host_staged:
+        pa = torch.empty(1 << 30, dtype=torch.uint8, device=dev)
+        pb = torch.empty(1 << 30, dtype=torch.uint8, device=dev)
+        pa.zero_(), pb.zero_()
+        probes = {name + "_GB/s": ep.ep_probe_bandwidth(kind, pb, pa, 1 << 30, iters=8)
+                  for name, kind in [("read", ep.PROBE_READ), ("write", ep.PROBE_WRITE), ("copy", ep.PROBE_COPY)]}
+        probes["what"] = "ep_probe_bandwidth, 1 GiB, best of 8; copy counts read + write bytes"
+        del pa, pb
+
     if rank != 0:
         rep.close()
         return
@@ -529,9 +540,12 @@ def main():
     dis_gbs = alg["dispatch"] / (dis_ms * 1e-3) / 1e9
 
     def roof(achieved, name):
-        return {"bound": "hbm", "kernel": name, "achieved": achieved, "peak": peak, "peak_kind": peak_kind + " copy peak",
-                "unit": "GB/s", "frac": achieved / peak, "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS,
-                "traffic": NCU_TRAFFIC_BYTES.get((cfg.name, name))}
+        r = {"bound": "hbm", "kernel": name, "achieved": achieved, "peak": peak, "peak_kind": peak_kind + " copy peak",
+             "unit": "GB/s", "frac": achieved / peak, "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS,
+             "traffic": NCU_TRAFFIC_BYTES.get((cfg.name, name))}
+        if probes:
+            r["frac_of_own_copy_probe"] = achieved / probes["copy_GB/s"]
+        return r
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -548,6 +562,7 @@ def main():
         },
         "roofline": roof(com_gbs, "combine_rows_kernel"),
         "roofline_dispatch": roof(dis_gbs, "dispatch_rows_kernel"),
+        "probes": probes,
         "clocks": clocks.summary(),
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": e2e_ms / n_e2e, "steps": args.e2e_steps,
