@@ -153,6 +153,31 @@ def test_layout_on_many_random_shapes():
         assert ep.ep_status(lay.status) == ref.status, (trial, T, K, E, R)
 
 
+def test_layout_halves_on_many_random_shapes():
+    """The two halves of the layout, called one after the other on the same workspace, over batch sizes
+    around every switch of the launch plan (one CTA, one cluster, many CTAs, larger tiles)."""
+    rng = np.random.default_rng(12)
+    sizes = [1, 30, 33, 1000, 1024, 1025, 2047, 3000, 4097, 8192, 9000, 20000, 32768, 33000, 50000]
+    for trial, tokens in enumerate(sizes):
+        R = int(rng.choice([1, 2, 4, 8, 64] if trial % 5 == 4 else [1, 2, 4, 8]))
+        T = max(R, tokens - tokens % R)
+        E = R * int(rng.choice([1, 4, 32]))
+        K = int(rng.integers(1, min(8, E) + 1))
+        idx = rng.integers(0, E, size=(T, K)).astype(np.int32)
+        if trial % 3 == 1:
+            idx[rng.random((T, K)) < 0.2] = -1
+        if trial % 4 == 2:
+            idx[int(rng.integers(0, T)), 0] = -5
+        ref = oracle.layout(idx, E, R)
+        idx_d = torch.from_numpy(idx).cuda()
+        lay = ep.alloc_layout(T, K, E, R, fill=-7)
+        ws = torch.empty(max(16, ep.ep_layout_workspace_bytes(T, K, E, R)), dtype=torch.uint8, device="cuda")
+        ep.ep_layout_ranks(idx_d, E, R, lay, ws)
+        ep.ep_layout_pairs(idx_d, E, R, lay, ws)
+        assert_layout_equal(lay, ref)
+        assert ep.ep_status(lay.status) == ref.status, (T, K, E, R)
+
+
 @pytest.mark.parametrize("name", ["C1", "C3", "C4"])
 def test_layout_halves_on_two_streams_equal_the_whole(name):
     """ep_layout_ranks and ep_layout_pairs, each on its own stream with its own workspace, fill
