@@ -136,8 +136,9 @@ int ep_layout_pairs(const ep_shape_t *shape, const int32_t *topk_idx, const ep_l
  * provides topk_idx and every output array.
  *
  *   - Limit: the scratch a shape needs is ep_layout_workspace_bytes(shape): 16
- *     bytes for batches of up to 2048 tokens, else 4*(E+R+1) bytes per CTA of
- *     8 token tiles, at most 128 CTAs (34 KB for T=8192, E=256, R=8). Shapes
+ *     bytes while the batch fits one thread-block cluster (2048 tokens, fewer
+ *     when large E or K shrink the CTA), else 4*(E+R+1) bytes per CTA, at most
+ *     128 CTAs (34 KB for T=8192, E=256, R=8). Shapes
  *     that need more than the array holds return EP_ERR_STATIC_SCRATCH and
  *     enqueue nothing.
  *   - First call on a device: looks up the array's device address (once per
@@ -180,8 +181,9 @@ int ep_combine(const ep_shape_t *shape, const void *out, int64_t out_rows, const
                const float *topk_weights, void *y, int32_t *status, void *stream);
 
 /*
- * Local grouping by expert (Section 4.3: "groups the tokens by the experts it
- * owns", a permutation that stays on the SMs): grouped[p] = recv[pair_row[p]]
+ * Local grouping by expert (Section 4.3: the receiver reorders what it received
+ * by the experts it owns, a permutation that stays on the SMs):
+ * grouped[p] = recv[pair_row[p]]
  * for p < P, where P is read on the device from expert_offsets[E]. grouped is
  * [grouped_capacity_rows][H] bf16 (device); entries p >= capacity are skipped
  * with EP_STATUS_CAPACITY.
@@ -192,7 +194,8 @@ int ep_group(const ep_shape_t *shape, const void *recv, int64_t recv_rows, const
 
 /*
  * Combine with partial outputs (Section 2.1, "Communication patterns of dispatch
- * and combine": the All-to-Allv form returns "partial outputs"): every rank
+ * and combine": in the All-to-Allv form what returns to the owner is one partial
+ * output per rank the token reached): every rank
  * first sums, per token it received, the weighted outputs of its own experts
  * into one row of `partial` (receive space, [partial_capacity_rows][H] bf16):
  *   partial[recv_slot[t][k]] = bf16( fp32 fma chain over the k' (ascending) that
@@ -242,8 +245,8 @@ int ep_dispatch_copy_engine(const ep_shape_t *shape, const void *x, const int32_
 
 /*
  * Host-staged round trip with separate upload and download streams (Section
- * 4.3: "uploads on one stream, downloads on another", chunked so that both
- * directions of the host link are busy; Section 4.4: two alternating bounce
+ * 4.3: uploads and downloads are issued on two different streams and cut into
+ * chunks so that both directions of the host link are busy; Section 4.4: two alternating bounce
  * buffers). Packs the receive rows into `staging` (device) with the dispatch
  * kernel on stream_up, copies them chunk by chunk to the bounce buffer
  * (pinned host, 2 * staging_capacity_rows rows: half `round & 1` is used) and

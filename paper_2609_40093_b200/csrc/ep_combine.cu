@@ -11,8 +11,6 @@
 // T=8192, H=7168, K=8). Small CTAs (128 threads, 63 registers, eight
 // resident per SM) measured 5 % faster alone than 448-thread groups with two
 // columns per thread (165 vs 175 us at T=8192, H=7168, K=8).
-#include <cstdlib>
-
 #include "ep_common.cuh"
 
 namespace ep {
@@ -156,13 +154,7 @@ int launch_combine(const ep_shape_t &s, const void *out, int64_t out_rows, const
     const int T = s.num_tokens, K = s.top_k, vpr = s.hidden / 8;
     const uint4 *o = static_cast<const uint4 *>(out);
     uint4 *yd = static_cast<uint4 *>(y);
-    int G = vpr <= 64 ? 32 : (vpr <= 256 ? 64 : 128);
-#ifdef EP_TUNING
-    if (const char *e = getenv("EP_TUNE_COMBINE")) {      // thread-group override, tuning builds only
-        const int v = atoi(e);
-        if (v == 32 || v == 64 || v == 128) G = v;
-    }
-#endif
+    const int G = vpr <= 64 ? 32 : (vpr <= 256 ? 64 : 128);
     if (G == 32)
         combine_rows_kernel<32><<<ceil_div(T, kBlock / 32), kBlock, 0, stream>>>(o, out_rows, slot, weights, yd, T, K, vpr, status);
     else if (G == 64)

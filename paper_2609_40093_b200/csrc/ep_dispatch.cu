@@ -4,9 +4,6 @@
 // destination row. Each warp finds its row's distinct destinations by itself
 // (K <= 32 slots, one per lane, duplicates dropped with a warp match), so there
 // is no shared memory and no block-wide barrier.
-#include <cstdio>
-#include <cstdlib>
-
 #include "ep_common.cuh"
 
 namespace ep {
@@ -20,7 +17,7 @@ struct RowPlan {
     int G, U, block, rows_per_block;
 };
 
-RowPlan plan_rows(int vec_per_row, const char *tune_env)
+RowPlan plan_rows(int vec_per_row)
 {
     RowPlan p;
     // two vectors per thread, up to 512 threads per row (measured: the row movers are HBM-bound for any
@@ -28,15 +25,6 @@ RowPlan plan_rows(int vec_per_row, const char *tune_env)
     int G = ceil_div(ceil_div(vec_per_row, 2), 32) * 32, U = 2;
     if (G > 512) G = 512;
     if (vec_per_row <= 32) U = 1;
-#ifdef EP_TUNING
-    if (const char *e = getenv(tune_env)) {      // "G,U" override, tuning builds only
-        int g = 0, u = 0;
-        if (sscanf(e, "%d,%d", &g, &u) == 2 && g >= 32 && g % 32 == 0 && (u == 1 || u == 2 || u == 4 || u == 8) &&
-            g <= (u == 8 ? 256 : (u == 4 ? 512 : 1024))) { G = g; U = u; }
-    }
-#else
-    (void)tune_env;
-#endif
     p.G = G;
     p.U = U;
     p.rows_per_block = G >= kMinBlock ? 1 : kMinBlock / G;
@@ -168,54 +156,6 @@ permute_rows_kernel(const uint4 *__restrict__ src, long long src_rows, const int
     }
 }
 
-#ifdef EP_TUNING
-// Experimental (tuning builds only): one warp per token; the row travels global -> shared -> every
-// destination as 1-D bulk copies (cp.async.bulk, no multicast), completion through an mbarrier with a
-// bounded wait.
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__global__ void __launch_bounds__(32)
-dispatch_bulk_kernel(const char *__restrict__ x, const int32_t *__restrict__ recv_slot, char *recv, int T, int K,
-                     uint32_t row_bytes, long long capacity_rows, int32_t *status)
-{
-    extern __shared__ __align__(128) char row_s[];
-    __shared__ __align__(8) unsigned long long bar;
-    const int lane = threadIdx.x, t = blockIdx.x;
-    if (t >= T) return;
-    int32_t slot = lane < K ? __ldg(recv_slot + (size_t)t * K + lane) : -1;
-    if (lane == 0) {
-        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&bar)));
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(&bar)), "r"(row_bytes) : "memory");
-        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(smem_u32(row_s)),
-                     "l"(x + (size_t)t * row_bytes), "r"(row_bytes), "r"(smem_u32(&bar))
-                     : "memory");
-    }
-    if (slot >= capacity_rows) {
-        flag_status(status, EP_STATUS_CAPACITY);
-        slot = -1;
-    }
-    const unsigned same = __match_any_sync(kFullMask, slot);
-    const unsigned todo = __ballot_sync(kFullMask, slot >= 0 && (same & lanemask_lt()) == 0);
-    __syncwarp();
-    bool ok = false;
-    for (int it = 0; it < (1 << 20) && !ok; ++it) {           // bounded wait for the row to land
-        uint32_t done;
-        asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], 0; selp.u32 %0,1,0,p; }"
-                     : "=r"(done) : "r"(smem_u32(&bar)) : "memory");
-        ok = done != 0;
-    }
-    if (!ok) {
-        if (lane == 0) flag_status(status, EP_STATUS_TIMEOUT);
-        return;
-    }
-    if ((todo >> lane) & 1u)                                    // each distinct destination: one bulk store
-        asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(recv + (size_t)slot * row_bytes),
-                     "r"(smem_u32(row_s)), "r"(row_bytes) : "memory");
-    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-    asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // shared memory stays valid until the copies have read it
-}
-#endif
 
 }  // namespace
 
@@ -224,7 +164,7 @@ int launch_permute(int hidden, const void *src, int64_t src_rows, const int32_t 
 {
     if (n <= 0) return EP_OK;
     const int vpr = hidden / 8;
-    const RowPlan p = plan_rows(vpr, "EP_TUNE_GROUP");
+    const RowPlan p = plan_rows(vpr);
     const unsigned grid = (unsigned)((n + p.rows_per_block - 1) / p.rows_per_block);
     const uint4 *s4 = static_cast<const uint4 *>(src);
     uint4 *d4 = static_cast<uint4 *>(dst);
@@ -242,19 +182,8 @@ int launch_dispatch(const ep_shape_t &s, const void *x, const int32_t *recv_slot
     const int T = s.num_tokens, K = s.top_k, vpr = s.hidden / 8;
     const uint4 *xs = static_cast<const uint4 *>(x);
     uint4 *rd = static_cast<uint4 *>(recv);
-    const RowPlan p = plan_rows(vpr, "EP_TUNE_DISPATCH");
+    const RowPlan p = plan_rows(vpr);
     const int grid = ceil_div(T, p.rows_per_block);
-#ifdef EP_TUNING
-    if (getenv("EP_TUNE_DISPATCH_BULK")) {
-        const uint32_t row_bytes = (uint32_t)vpr * 16;
-        static bool attr = false;
-        if (!attr) { cudaFuncSetAttribute(dispatch_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024); attr = true; }
-        dispatch_bulk_kernel<<<T, 32, row_bytes, stream>>>(static_cast<const char *>(x), recv_slot, static_cast<char *>(recv), T, K,
-                                                           row_bytes, capacity_rows, status);
-        EP_LAUNCH_CHECK(1);
-        return EP_OK;
-    }
-#endif
     switch (p.U) {
     case 1: dispatch_rows_kernel<1><<<grid, p.block, 0, stream>>>(xs, recv_slot, rd, T, K, vpr, p.G, capacity_rows, status); break;
     case 2: dispatch_rows_kernel<2><<<grid, p.block, 0, stream>>>(xs, recv_slot, rd, T, K, vpr, p.G, capacity_rows, status); break;
@@ -273,7 +202,7 @@ int launch_group(const ep_shape_t &s, const void *recv, int64_t recv_rows, const
     const int vpr = s.hidden / 8;
     const uint4 *rs = static_cast<const uint4 *>(recv);
     uint4 *gd = static_cast<uint4 *>(grouped);
-    const RowPlan p = plan_rows(vpr, "EP_TUNE_GROUP");
+    const RowPlan p = plan_rows(vpr);
     const unsigned grid = (unsigned)((max_pairs + p.rows_per_block - 1) / p.rows_per_block);
     switch (p.U) {
     case 1: group_rows_kernel<1><<<grid, p.block, 0, stream>>>(rs, recv_rows, pair_row, n_pairs, gd, capacity_rows, vpr, p.G, status); break;

@@ -106,18 +106,8 @@ __device__ __forceinline__ int fdiv(int n, const FastDiv &f)
     return f.d == 1 ? n : (int)__umul64hi((uint64_t)(uint32_t)n, f.m);
 }
 
-// phase time stamps of the main kernel, compiled only with -DEP_LAYOUT_TIMING (never in the product build)
-#ifdef EP_LAYOUT_TIMING
-static long long *g_timing_buf = nullptr;
-#define EP_STAMP(i) do { if (a.dbg && threadIdx.x == 0) a.dbg[blockIdx.x * 16 + (i)] = clock64(); } while (0)
-#else
-#define EP_STAMP(i) do { } while (0)
-#endif
 
 struct LayoutArgs {
-#ifdef EP_LAYOUT_TIMING
-    long long *dbg;
-#endif
     const int32_t *idx;
     ep_layout_t out;
     int32_t *cta_part;  // [n_ctas][bins], global form only
@@ -255,10 +245,8 @@ __global__ void __launch_bounds__(kMaxWarpsSingle * 32) layout_assign_kernel(Lay
     const int tile = blockIdx.x * warps + warp;
     const unsigned lt = lanemask_lt();
 
-    EP_STAMP(0);
     count_tile<false>(a, run, ids, tile, lane);
     __syncthreads();
-    EP_STAMP(1);
     const bool ranks = a.parts & kPartRanks, pairs = a.parts & kPartPairs;
     for (int b = a.blo + threadIdx.x; b < a.bins; b += blockDim.x) {  // this CTA's total per bin
         int32_t mine = 0;
@@ -267,7 +255,6 @@ __global__ void __launch_bounds__(kMaxWarpsSingle * 32) layout_assign_kernel(Lay
     }
     if (a.mode == kModeCluster) cg::this_cluster().sync();           // every peer's cta_tot is written
     else if (a.mode == kModeGlobal) pdl_wait();                      // cta_part is complete and visible
-    EP_STAMP(2);
     // per bin: count in earlier CTAs and grand total (each thread reads the cta_tot entries it wrote itself)
     for (int b = a.blo + threadIdx.x; b < a.bins; b += blockDim.x) {
         int32_t before = 0, total = 0;
@@ -300,7 +287,6 @@ __global__ void __launch_bounds__(kMaxWarpsSingle * 32) layout_assign_kernel(Lay
     }
     if (a.mode == kModeCluster) cg::this_cluster().sync();           // peers are done with this CTA's shared memory
     else __syncthreads();
-    EP_STAMP(3);
     // one exclusive scan over [experts | ranks]: S[e] = expert offset, S[E + r] - S[E] = rank row offset
     block_exclusive_scan_smem(tot + a.blo, nb - a.blo, sh);
     const int32_t n_pairs = tot[a.E];                                // 0 when the scan started at the rank bins
@@ -323,7 +309,6 @@ __global__ void __launch_bounds__(kMaxWarpsSingle * 32) layout_assign_kernel(Lay
         }
     }
     __syncthreads();
-    EP_STAMP(4);
     if (tile >= a.n_tiles) return;
 
     // replay the tile in (t,k) order; run[bin] = next free slot of the bin
@@ -395,16 +380,11 @@ __global__ void __launch_bounds__(kMaxWarpsSingle * 32) layout_assign_kernel(Lay
             if (valid && (m >> lane) <= 1u) run[e] = first + __popc(m);   // highest lane of the group
             __syncwarp();
         }
-        EP_STAMP(5 + (tb - t0) / 32);
     }
 }
 
 }  // namespace
 }  // namespace ep
-
-#ifdef EP_LAYOUT_TIMING
-extern "C" void ep_debug_set_timing_buffer(long long *p) { ep::g_timing_buf = p; }
-#endif
 
 extern "C" size_t ep_layout_workspace_bytes(const ep_shape_t *shape)
 {
@@ -456,9 +436,6 @@ int run_layout(const ep_shape_t *shape, const int32_t *topk_idx, const ep_layout
     a.mode = plan.mode;
     a.parts = parts;
     a.blo = pairs ? 0 : E;
-#ifdef EP_LAYOUT_TIMING
-    a.dbg = g_timing_buf;
-#endif
 
     static std::atomic<bool> attr_done[64] = {};       // per device: dynamic shared memory limit raised
     int dev = 0;
@@ -565,7 +542,7 @@ extern "C" int ep_layout_static(const ep_shape_t *shape, const int32_t *topk_idx
     void *scratch = nullptr;
     rc = ep::static_scratch_address(&scratch);
     if (rc != EP_OK) return rc;
-    // pass 1 rewrites every scratch word it later reads (including the CTA ticket),
-    // so whatever the previous call left in the array needs no clearing
+    // the counting kernel rewrites every cta_part word (bins blo..bins of every CTA) that the
+    // assign kernel reads, so whatever the previous call left in the array needs no clearing
     return ep_layout(shape, topk_idx, out, scratch, EP_LAYOUT_STATIC_SCRATCH_BYTES, stream);
 }

@@ -151,25 +151,136 @@ def test_dense_formulation_volumes_and_values():
     np.testing.assert_array_equal(y[single], y2[single])
 
 
+def _dense_exact(out_f, idx, pair_slot, w, E, R):
+    """Dense reduce-scatter on exact rationals with explicit roundings (tiny inputs): per rank an fp32
+    fma chain over the k (ascending) whose expert lives there, one bf16 rounding of what the rank places
+    in its dense buffer, then the owner's fp32 sum of the R placed values in the order r = 0..R-1."""
+    T, K = idx.shape
+    H = out_f.shape[1]
+    El = E // R
+    dense = np.zeros((R, T, H))
+    y = np.zeros((T, H))
+    for t in range(T):
+        for h in range(H):
+            total = Fraction(0)
+            for r in range(R):
+                acc = Fraction(0)
+                for k in range(K):
+                    if 0 <= idx[t, k] < E and idx[t, k] // El == r:
+                        acc = brute.round_f32(Fraction(float(w[t, k])) * Fraction(float(out_f[pair_slot[t, k], h])) + acc)
+                placed = brute.round_bf16(acc)
+                dense[r, t, h] = float(placed)
+                total = brute.round_f32(total + placed)
+            y[t, h] = float(brute.round_bf16(total))
+    return dense, y
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2])
+def test_dense_reduce_scatter_against_exact_rationals(seed):
+    """8 experts on 4 ranks, 4 distinct picks per token: every token reaches at least two ranks and most
+    reach three or four, so the owner's sum has several terms that are not bf16 numbers before placing."""
+    cfg, idx, w, x, lay, out = _case(8, 6, 8, 4, 4, cid=86, seed=seed)
+    assert max(len(set((idx[t] // 2).tolist())) for t in range(cfg.T)) >= 3
+    dense, y = oracle.dense_reduce_scatter(idx, out, lay.pair_slot, w, cfg.E, cfg.R)
+    want_dense, want_y = _dense_exact(inputs.bf16_bits_to_f32(out), idx, lay.pair_slot, w, cfg.E, cfg.R)
+    np.testing.assert_array_equal(inputs.bf16_bits_to_f32(dense).astype(np.float64).reshape(cfg.R, cfg.T, cfg.H),
+                                  want_dense)
+    np.testing.assert_array_equal(inputs.bf16_bits_to_f32(y).astype(np.float64), want_y)
+
+
+def test_dense_reduce_scatter_sums_ranks_in_ascending_order_and_after_rounding():
+    """Three ranks hold big, -big and small: summed in the order r = 0, 1, 2 the small term survives;
+    any order that adds small to a big term first loses it. Then a rank whose fp32 partial is not a
+    bf16 number: the owner must add what was placed (rounded), not the unrounded accumulator."""
+    E, R, H = 3, 3, 1
+    out = inputs.to_bf16_bits(np.array([[2.0 ** 20], [2.0 ** 20], [2.0 ** -6]], dtype=np.float32))
+    w = np.array([[1.0, -1.0, 1.0]] * 3, dtype=np.float32)
+    idx = np.array([[0, 1, 2]] * 3, dtype=np.int32)                 # pick k sits on rank k
+    pair_slot = np.array([[0, 1, 2]] * 3, dtype=np.int32)
+    dense, y = oracle.dense_reduce_scatter(idx, out, pair_slot, w, E, R)
+    assert (inputs.bf16_bits_to_f32(y) == 2.0 ** -6).all()
+    idx2 = np.array([[2, 1, 0]] * 3, dtype=np.int32)                # big on rank 2, -big on rank 1, small on rank 0
+    w2 = np.array([[1.0, -1.0, 1.0]] * 3, dtype=np.float32)
+    out2 = inputs.to_bf16_bits(np.array([[2.0 ** 20], [2.0 ** 20], [2.0 ** -6]], dtype=np.float32))
+    pair2 = np.array([[0, 1, 2]] * 3, dtype=np.int32)               # k=0 -> big (rank 2), k=1 -> -big (rank 1), k=2 -> small (rank 0)
+    _, y2 = oracle.dense_reduce_scatter(idx2, out2, pair2, w2, E, R)
+    assert (inputs.bf16_bits_to_f32(y2) == 0.0).all()               # small + (-big) = -big; -big + big = 0
+    # rank 0 holds 1 + 2^-10 in fp32 (two picks), which it places as bf16 1.0; rank 1 holds -1
+    E, R = 4, 2
+    out3 = inputs.to_bf16_bits(np.array([[1.0], [2.0 ** -10], [1.0]], dtype=np.float32))
+    idx3 = np.array([[0, 1, 2]] * 2, dtype=np.int32)                # experts 0, 1 on rank 0; expert 2 on rank 1
+    w3 = np.array([[1.0, 1.0, -1.0]] * 2, dtype=np.float32)
+    pair3 = np.array([[0, 1, 2]] * 2, dtype=np.int32)
+    dense3, y3 = oracle.dense_reduce_scatter(idx3, out3, pair3, w3, E, R)
+    assert (inputs.bf16_bits_to_f32(dense3).ravel() == np.array([1.0, 1.0, -1.0, -1.0])).all()
+    assert (inputs.bf16_bits_to_f32(y3) == 0.0).all()               # 2^-10 would survive an unrounded sum
+
+
+def _ring_allgather_bytes(N, S):
+    """Replays the ring schedule over a host bounce buffer (no P2P): at each of N-1 steps every GPU
+    uploads the shard it obtained last and downloads the one its predecessor uploaded. Returns the
+    bytes per GPU over the host link and checks that every GPU ends up holding every shard."""
+    holds = [{g} for g in range(N)]
+    last = list(range(N))
+    moved = [0] * N
+    for _ in range(N - 1):
+        sent = list(last)
+        for g in range(N):
+            moved[g] += S                                            # upload of the shard obtained last
+        for g in range(N):
+            got = sent[(g - 1) % N]
+            moved[g] += S                                            # download from the predecessor
+            holds[g].add(got)
+            last[g] = got
+    assert all(h == set(range(N)) for h in holds)
+    assert len(set(moved)) == 1
+    return moved[0]
+
+
 @pytest.mark.parametrize("N", [2, 4, 6])
 def test_paper_traffic_formulas(N):
-    """Section 4.2: per-GPU PCIe volume of an all-gather of shards S: ring 2(N-1)S,
-    single-step N*S, ratio 2(N-1)/N (1 at N=2; 10S -> 6S at N=6); reduce-scatter with GPU
-    reduction 2(N-1)S, with CPU reduction N*S. Counted on the dense oracle's buffers."""
-    T, H = 12 * N, 16
-    S = (T // N) * H * 2                                               # one rank's shard in bytes
-    x = inputs.make_x(inputs.custom_config(T, H, N, 1, N, config_id=85))
-    g = oracle.dense_allgather(x, N)
-    per_rank_rows = g.shape[0] // N
-    single_step = S + (per_rank_rows - T // N) * H * 2                 # upload own shard once, download the others
-    assert single_step == N * S
-    ring = sum(2 * S for _ in range(N - 1))                            # one upload and one download per step
+    """Section 4.2, per-GPU volume over the host link with shards of S bytes: ring all-gather 2(N-1)S,
+    single-step all-gather N*S, ratio 2(N-1)/N (1 at N=2; 10S -> 6S at N=6); reduce-scatter with GPU
+    reduction 2(N-1)S, with CPU reduction N*S. The single-step volumes are counted on the dense oracle's
+    buffers (which rows of a rank's block come from, or go to, another rank), the ring by replaying its
+    schedule; neither count uses the formula it is compared with."""
+    T, H, K = 12 * N, 16, 2
+    Tr = T // N
+    row = 2 * H
+    S = Tr * row                                                     # one rank's shard in bytes
+    cfg = inputs.custom_config(T, H, 2 * N, K, N, config_id=85)
+    d = inputs.make_inputs(cfg)
+    x, idx, w = d["x"], d["topk_idx"], d["topk_weights"]
+    g = oracle.dense_allgather(x, N).reshape(N, T, H)
+    owner = np.arange(T) // Tr
+    for r in range(N):
+        written = np.flatnonzero((g[r] != 0).any(axis=1))            # the wrapper starts from zeros; no row of x is all zero
+        remote = written[owner[written] != r]
+        download = remote.size * row                                 # rows of other ranks' shards that rank r reads back
+        sources = {int(s) for s in owner[remote]}
+        assert sources == set(range(N)) - {r}
+        upload = np.unique(x[owner == r], axis=0).shape[0] * row     # rank r's own shard goes up once, whoever reads it
+        assert upload == S and download == (N - 1) * S
+        assert upload + download == N * S
+    ring = _ring_allgather_bytes(N, S)
     assert ring == 2 * (N - 1) * S
-    assert Fraction(ring, single_step) == Fraction(2 * (N - 1), N)
+    assert Fraction(ring, N * S) == Fraction(2 * (N - 1), N)
     if N == 2:
-        assert ring == single_step
+        assert ring == N * S
     if N == 6:
-        assert (ring // S, single_step // S) == (10, 6)
-    rs_gpu = (N - 1) * S + (N - 1) * S                                 # upload N-1 blocks, download N-1 blocks
-    rs_cpu = (N - 1) * S + S
-    assert rs_gpu == 2 * (N - 1) * S and rs_cpu == N * S
+        assert (ring // S, N * S // S) == (10, 6)
+    # reduce-scatter: rank r's dense block holds one row per source token; the rows of tokens another rank
+    # owns are the blocks it uploads, the rows other ranks hold for its own tokens are what it downloads
+    lay = oracle.layout(idx, cfg.E, N)
+    out = inputs.make_out(cfg, lay.n_pairs)
+    dense, _ = oracle.dense_reduce_scatter(idx, out, lay.pair_slot, w, cfg.E, N)
+    dense = dense.reshape(N, T, H)
+    assert dense.shape[1] == T                                       # a full source-ordered block per rank, whatever the routing
+    for r in range(N):
+        up_rows = int((owner != r).sum())                            # rows of rank r's block destined for other ranks
+        down_rows = sum(int((owner == r).sum()) for q in range(N) if q != r)
+        assert up_rows * row == (N - 1) * S and down_rows * row == (N - 1) * S
+        assert (up_rows + down_rows) * row == 2 * (N - 1) * S        # GPU reduction: same volume as the ring
+        assert up_rows * row + int((owner == r).sum()) * row == N * S   # CPU reduction: one reduced block comes down
+    # the routed form moves only the rows a rank needs: never more than the dense R*T, never more than T*min(K,R)
+    assert lay.n_recv <= T * min(K, N) <= N * T

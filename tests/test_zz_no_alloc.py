@@ -10,12 +10,12 @@ produces: leftovers of the first call must not leak into the second. This file
 sorts last so that a run that stops at the first failure has already covered
 everything else; it does not depend on any other test having run.
 """
-import ctypes
-
 import numpy as np
 import pytest
 import torch
 
+import oracle
+from gpu_util import assert_layout_equal
 from paper_2609_40093_b200 import ep, inputs
 
 pytestmark = pytest.mark.gpu
@@ -48,6 +48,7 @@ def test_static_scratch_layout_matches_ep_layout_on_two_calls_in_a_row():
         ep.ep_layout_static(idx, cfg.E, cfg.R, out=got)
         torch.cuda.synchronize()
         _same(got, want)
+        assert_layout_equal(got, oracle.layout(inputs.make_topk_idx(cfg), cfg.E, cfg.R))
     # a table with masked and out-of-range ids: the status word travels the same way
     cfg = inputs.custom_config(512, 8, 64, 4, 8, config_id=77)
     idx_h = inputs.make_topk_idx(cfg)
@@ -61,7 +62,8 @@ def test_static_scratch_layout_matches_ep_layout_on_two_calls_in_a_row():
 
 
 def test_static_scratch_rejects_shapes_beyond_its_limit():
-    # E = 4096 experts over 32768 tokens needs ~16 MiB of scratch: refused, nothing enqueued
+    # E = 4096 experts and R = 64 ranks over 32768 tokens: 128 CTAs x 4161 counters x 4 bytes, about
+    # 2.1 MB of scratch, twice what the fixed array holds: refused, nothing enqueued
     T, K, E, R = 32768, 2, 4096, 64
     assert ep.ep_layout_workspace_bytes(T, K, E, R) > ep.ep_layout_static_scratch_bytes()
     idx = torch.zeros(T, K, dtype=torch.int32, device="cuda")
@@ -71,3 +73,26 @@ def test_static_scratch_rejects_shapes_beyond_its_limit():
     assert err.value.code == -5
     torch.cuda.synchronize()
     assert int(out.expert_offsets[-1]) == -5 and int(out.status[0]) == -5      # outputs untouched
+
+
+def test_static_scratch_calls_allocate_nothing_and_may_follow_each_other_without_a_sync():
+    """What the entry point is for: after the first call on the device (which looks the array up) no
+    call changes the amount of free device memory, and two calls on different routing tables queued
+    on one stream with no host synchronisation between them both come out right (the second call
+    reuses the scratch the first one left behind; stream order is all that separates them)."""
+    a = inputs.custom_config(40000, 8, 16, 2, 8, config_id=78)
+    b = inputs.custom_config(24000, 8, 64, 4, 8, routing="zipf", config_id=76)
+    tables = [torch.from_numpy(inputs.make_topk_idx(c)).cuda() for c in (a, b)]
+    outs = [ep.alloc_layout(c.T, c.K, c.E, c.R, fill=-5) for c in (a, b)]
+    ep.ep_layout_static(tables[0], a.E, a.R, out=outs[0])                # first call: address look-up
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info()
+    for _ in range(3):
+        for c, idx, out in zip((a, b), tables, outs):
+            ep.ep_layout_static(idx, c.E, c.R, out=out)                   # no synchronisation in between
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before
+    for c, out in zip((a, b), outs):
+        assert_layout_equal(out, oracle.layout(inputs.make_topk_idx(c), c.E, c.R))
+        assert ep.ep_status(out.status) == 0
