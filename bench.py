@@ -5,9 +5,12 @@
 
 One step = layout -> dispatch -> combine over one batch of seeded synthetic routing
 (combine reads T*K independent expert-output rows in the pair space). Prints ONE
-JSON line on rank 0. With N > 1 every rank runs an independent replica of the
-workload (the path has no exchange between GPUs); the time is the max over ranks.
-`--impl reference` times the CPU oracle on the host cores instead.
+JSON line on rank 0. The headline workload is C4 (the largest configuration); the
+same line carries, under `configs`, the step and per-kernel figures of the other
+configurations (C1, C2, C3 and the host-staged C5 with its host-link roofline).
+With N > 1 every rank runs an independent replica of the workload (the path has no
+exchange between GPUs); the time is the max over ranks.
+`--impl reference` times the CPU oracle on the host cores on the same batch.
 """
 from __future__ import annotations
 
@@ -17,6 +20,7 @@ import os
 import sys
 import threading
 import time
+from concurrent.futures import ThreadPoolExecutor
 
 ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
@@ -29,10 +33,11 @@ METRIC = "ep_layout_dispatch_combine_tokens_per_s"
 UNIT = "tokens/s"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
-# DRAM bytes per launch of the dominant kernel from the committed ncu capture
-# (profiles/): filled in per workload once measured, else null.
+# DRAM bytes per launch of the dominant kernels from the committed ncu captures (profiles/).
 NCU_TRAFFIC_BYTES = {("C4", "combine_rows_kernel"): 1038.7e6, ("C4", "dispatch_rows_kernel"): 680.8e6}
 L2_BYTES = 126e6
+CONTEXT = ("paper reports 2.00x (dispatch) / 1.53x (combine) over NCCL for its dense all-gather/"
+           "reduce-scatter on RTX 4090/5090 PCIe boxes; no number for the routing-aware path")
 
 
 class L2Flush:
@@ -51,133 +56,9 @@ class L2Flush:
         torch.sum(self.r)
 
 
-def launches_per_step(ep, step):
-    """Kernels one direct (non-graph) step launches, counted by the library."""
-    n0 = ep.ep_launch_count()
-    step()
-    torch.cuda.synchronize()
-    return ep.ep_launch_count() - n0
-
-
-def time_variants(ep, cfg, idx, w, x, out, lay, n_recv, n_pairs, dev, iters=20):
-    """Median device time of the variants around the path on the same batch: local grouping,
-    expanded dispatch, combine with per-rank partial outputs, dense all-gather / reduce-scatter."""
-    T, K, H, E, R = cfg.T, cfg.K, cfg.H, cfg.E, cfg.R
-    row = 2 * H
-    flush = L2Flush(dev)
-    recv = torch.empty(max(1, n_recv), H, dtype=torch.bfloat16, device=dev)
-    ep.ep_dispatch(x, lay.recv_slot, recv, E, R)
-    y = torch.empty(T, H, dtype=torch.bfloat16, device=dev)
-    res = {"rows": {"routed_receive": n_recv, "pairs": n_pairs, "dense": R * T}}
-
-    def timed(fn, nbytes):
-        ts = []
-        for _ in range(iters + 2):
-            flush()
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record()
-            fn()
-            b.record()
-            torch.cuda.synchronize()
-            ts.append(a.elapsed_time(b))
-        ms = float(np.median(ts[2:]))
-        return {"us": ms * 1e3, "GB/s": nbytes / (ms * 1e-3) / 1e9, "bytes": nbytes}
-
-    grouped = torch.empty(max(1, n_pairs), H, dtype=torch.bfloat16, device=dev)
-    res["group (recv -> pair rows)"] = timed(lambda: ep.ep_group(recv, lay, grouped, E, R), 2 * row * n_pairs + 4 * n_pairs)
-    res["expanded dispatch (x -> pair rows)"] = timed(lambda: ep.ep_dispatch(x, lay.pair_slot, grouped, E, R),
-                                                      row * T + row * n_pairs + 4 * T * K)
-    del grouped
-    partial = torch.empty(max(1, n_recv), H, dtype=torch.bfloat16, device=dev)
-    res["combine with partial outputs (2 kernels)"] = timed(
-        lambda: ep.ep_combine_partial(out, lay, w, partial, y, E, R),
-        row * n_pairs + 2 * row * n_recv + row * T + 16 * T * K)
-    del partial
-    gathered = torch.empty(R * T, H, dtype=torch.bfloat16, device=dev)
-    res["dense all-gather"] = timed(lambda: ep.ep_dense_allgather(x, gathered, K, E, R), row * T + row * R * T)
-    if R <= 32:
-        res["dense reduce-scatter (2 kernels)"] = timed(
-            lambda: ep.ep_dense_reduce_scatter(idx, out, lay.pair_slot, w, gathered, y, E, R),
-            row * n_pairs + 2 * row * R * T + row * T + 12 * T * K)
-    del gathered, flush
-    return res
-
-
-def host_staged_arms(ep, cfg, x, lay, recv_host, dev, iters=10):
-    """Receive buffer in mapped pinned host memory: (i) the dispatch kernel stores straight
-    into it; (ii) dispatch packs into device staging and the copy engine moves each rank's
-    partition; plus the host-link probe both are measured against."""
-    E, R = cfg.E, cfg.R
-    n_recv = int(lay.rank_row_offsets[-1])
-    row = 2 * cfg.H
-    staging = torch.empty(recv_host.shape[0], cfg.H, dtype=torch.bfloat16, device=dev)
-    probe_src = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
-    probe_dst = torch.empty(256 << 20, dtype=torch.uint8).pin_memory()
-    d2h = ep.ep_probe_bandwidth(ep.PROBE_MEMCPY, probe_dst, probe_src, 256 << 20, iters=10)
-    h2d = ep.ep_probe_bandwidth(ep.PROBE_MEMCPY, probe_src, probe_dst, 256 << 20, iters=10)
-
-    def timed(fn):
-        best = 1e30
-        for _ in range(iters + 1):
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record()
-            fn()
-            b.record()
-            torch.cuda.synchronize()
-            best = min(best, a.elapsed_time(b))
-        return best
-
-    def arm_kernel():
-        ep.ep_dispatch(x, lay.recv_slot, recv_host, E, R)
-
-    offs_pinned = torch.zeros(R + 1, dtype=torch.int32).pin_memory()
-
-    def arm_copy_known():           # the offsets first travel to the host: one small copy and a stream sync, timed
-        offs_pinned.copy_(lay.rank_row_offsets, non_blocking=True)
-        torch.cuda.current_stream().synchronize()
-        ep.ep_dispatch_copy_engine(x, lay.recv_slot, staging, recv_host, E, R, rank_row_offsets_host=offs_pinned)
-
-    def arm_copy_blind():           # no count reaches the host: one copy of the worst-case T*min(K,R) rows
-        ep.ep_dispatch_copy_engine(x, lay.recv_slot, staging, recv_host, E, R, rank_row_offsets_host=None)
-
-    res = {"host_link_d2h_GB/s": d2h, "host_link_h2d_GB/s": h2d, "rows": n_recv, "bytes_over_link": n_recv * row}
-    # round trip through the bounce buffer on two streams: all uploads then all downloads, or chunk-wise duplex
-    cap = recv_host.shape[0]
-    bounce = torch.empty(2 * cap, cfg.H, dtype=torch.bfloat16).pin_memory()
-    back = torch.empty(cap, cfg.H, dtype=torch.bfloat16, device=dev)
-    up, down = torch.cuda.Stream(), torch.cuda.Stream()
-    offs_host = lay.rank_row_offsets.cpu()
-    torch.cuda.synchronize()
-    trips = {}
-    for duplex, chunks in [(0, 1), (1, 1), (1, 2), (1, 4), (1, 8)]:
-        best = 1e30
-        for rnd in range(iters + 1):
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            a.record(down)
-            ep.ep_host_roundtrip(x, lay.recv_slot, offs_host, staging, bounce, back, E, R, round=rnd,
-                                 chunks_per_rank=chunks, duplex=bool(duplex), stream_up=up, stream_down=down)
-            b.record(down)
-            torch.cuda.synchronize()
-            best = min(best, a.elapsed_time(b))
-        trips[("duplex" if duplex else "serial") + f", {chunks} chunk(s) per rank"] = {
-            "us": best * 1e3, "GB/s_each_way": n_recv * row / (best * 1e-3) / 1e9, "tokens/s": cfg.T / (best * 1e-3)}
-    # cost of one completion check: the wait kernel on flags that are already posted
-    n_s = max(1, R - 1)
-    flags_dev = torch.full((64,), 3, dtype=torch.int32, device=dev)
-    flags_pin = torch.full((64,), 3, dtype=torch.int32).pin_memory()
-    waits = {}
-    for name, fl in [("flags in device memory", flags_dev), ("flags in pinned host memory", flags_pin)]:
-        waits[name] = {"us": timed(lambda: ep.ep_wait_senders(fl, n_s, 3, 100_000_000)) * 1e3, "senders": n_s}
-
-    res["roundtrip"] = trips
-    res["flag_wait_posted"] = waits
-    for name, fn, nbytes in [("kernel_store", arm_kernel, n_recv * row),
-                             ("copy_engine_per_rank", arm_copy_known, n_recv * row),
-                             ("copy_engine_worst_case", arm_copy_blind, recv_host.shape[0] * row)]:
-        ms = timed(fn)
-        res[name] = {"us": ms * 1e3, "GB/s": nbytes / (ms * 1e-3) / 1e9, "useful_GB/s": n_recv * row / (ms * 1e-3) / 1e9,
-                     "frac_of_d2h_probe": n_recv * row / (ms * 1e-3) / 1e9 / d2h, "tokens/s": cfg.T / (ms * 1e-3)}
-    return res
+def stats_us(ms_values):
+    a = np.asarray(ms_values, dtype=np.float64) * 1e3
+    return {"us": float(a.mean()), "median_us": float(np.median(a)), "best_us": float(a.min())}
 
 
 def workload_text(cfg):
@@ -185,6 +66,24 @@ def workload_text(cfg):
                "burst": "uniform routing + 10% hot-expert burst on expert 0"}[cfg.routing]
     return (f"{cfg.name}: T={cfg.T} H={cfg.H} E={cfg.E} K={cfg.K} R={cfg.R}, {routing}, bf16 N(0,1) rows, "
             f"softmax weights" + (", receive buffer in mapped pinned host memory" if cfg.host_staged else ""))
+
+
+def step_bytes_estimate(cfg):
+    return 2 * cfg.H * (2 * cfg.T + cfg.T * min(cfg.K, cfg.R) + cfg.T * cfg.K)
+
+
+def is_small(cfg):
+    """The step's data could (partly) stay in L2 from one step to the next."""
+    return step_bytes_estimate(cfg) < 4 * L2_BYTES and not cfg.host_staged
+
+
+def config_object(cfg, world, n_recv, n_pairs):
+    """The `config` of the JSON line: a function of the workload alone, identical in both arms."""
+    l2 = ("step data would fit L2: before every timed step 256 MB are written and then another 256 MB read "
+          "(L2 left holding clean foreign lines); each step timed by its own event pair") if is_small(cfg) else \
+        "working set per step exceeds L2 several times over (no flush needed)"
+    return {"workload": workload_text(cfg), "parallelism": f"{world} independent replica(s)", "l2": l2,
+            "n_recv": int(n_recv), "n_pairs": int(n_pairs)}
 
 
 def measured_peak():
@@ -265,71 +164,414 @@ class ClockSampler:
                 "reasons": sorted(self.reasons), "samples": len(self.samples)}
 
 
-def cpu_oracle_step(oracle, idx, w, x, out):
-    lay = oracle.layout(idx, CPU_CFG.E, CPU_CFG.R)
+# --------------------------------------------------------------------------- CPU oracle legs
+
+def oracle_step(oracle, cfg, idx, w, x, out):
+    """One whole step of the oracle as it stands, one thread."""
+    lay = oracle.layout(idx, cfg.E, cfg.R)
     oracle.dispatch(x, lay.recv_slot, lay.n_recv)
     oracle.combine_f32(out, lay.pair_slot, w)
 
 
+def oracle_step_all_cores(oracle, pool, n_threads, cfg, idx, w, x, out):
+    """The same step with the token range cut statically into one contiguous part per thread for
+    dispatch and combine (independent per token once the slots exist); the layout stays serial.
+    The oracle's C functions are called unchanged on row slices; ctypes releases the GIL."""
+    lay = oracle.layout(idx, cfg.E, cfg.R)
+    T = cfg.T
+    cuts = [T * i // n_threads for i in range(n_threads + 1)]
+    recv = np.empty((max(1, lay.n_recv), cfg.H), dtype=np.uint16)
+    y = np.empty((T, cfg.H), dtype=np.uint16)
+    parts = [(a, b) for a, b in zip(cuts[:-1], cuts[1:]) if b > a]
+    list(pool.map(lambda ab: oracle.dispatch_into(x[ab[0]:ab[1]], lay.recv_slot[ab[0]:ab[1]], recv), parts))
+    list(pool.map(lambda ab: oracle.combine_f32_into(out, lay.pair_slot[ab[0]:ab[1]], w[ab[0]:ab[1]], y[ab[0]:ab[1]]),
+                  parts))
+
+
+def usable_cores():
+    try:
+        return len(os.sched_getaffinity(0))
+    except Exception:
+        return os.cpu_count() or 1
+
+
 def time_oracle(cfg, idx, w, x, out, min_seconds, max_steps):
-    """Times whole oracle steps (layout + dispatch + combine, one thread) on the given batch."""
+    """Whole oracle steps on the given batch: one thread, then all usable cores."""
     import oracle
-    global CPU_CFG
-    CPU_CFG = cfg
     oracle.build()
-    steps, t0 = 0, time.perf_counter()
-    while True:
-        cpu_oracle_step(oracle, idx, w, x, out)
-        steps += 1
-        el = time.perf_counter() - t0
-        if el >= min_seconds or steps >= max_steps:
-            return idx.shape[0] * steps / el, steps, el
+
+    def run(fn):
+        fn()                                            # page in
+        steps, t0 = 0, time.perf_counter()
+        while True:
+            fn()
+            steps += 1
+            el = time.perf_counter() - t0
+            if el >= min_seconds or steps >= max_steps:
+                return cfg.T * steps / el, steps, el
+
+    v1, n1, el1 = run(lambda: oracle_step(oracle, cfg, idx, w, x, out))
+    cores = usable_cores()
+    with ThreadPoolExecutor(max_workers=cores) as pool:
+        vn, nn, eln = run(lambda: oracle_step_all_cores(oracle, pool, cores, cfg, idx, w, x, out))
+    return {"value": v1, "unit": UNIT, "cores": 1, "kind": "oracle",
+            "sample": f"{n1} whole step(s) of the same {cfg.name} batch in {el1:.1f} s, one thread",
+            "all_cores": {"value": vn, "unit": UNIT, "cores": cores,
+                          "sample": f"{nn} whole step(s) of the same batch in {eln:.1f} s; layout serial, dispatch and "
+                                    f"combine split statically over {cores} threads by token range"},
+            "host_cores_available": os.cpu_count()}
 
 
 def run_reference(args, cfg):
-    """The CPU oracle as the reference arm: each step is the oracle on the first
-    `sample` tokens of the workload (all K picks, all R ranks)."""
+    """The CPU oracle as the reference arm, on the same batch and generators as the GPU arm: each step
+    is one whole oracle step (layout + dispatch + combine, one thread) over all T tokens."""
     from paper_2609_40093_b200 import inputs
     import oracle
-    global CPU_CFG
-    CPU_CFG = cfg
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     oracle.build()
-    sample = min(cfg.T, 1024)
-    sample -= sample % cfg.R
-    idx = inputs.make_topk_idx(cfg)[:sample]
-    w = inputs.make_topk_weights(cfg)[:sample]
-    sub = inputs.custom_config(sample, cfg.H, cfg.E, cfg.K, cfg.R, routing="uniform", config_id=cfg.config_id)
-    x = inputs.make_x(sub)
-    out = inputs.make_out(sub, sample * cfg.K)
-    # shrink the sample if the requested number of steps would run for more than ~3 minutes
-    t0 = time.perf_counter()
-    cpu_oracle_step(oracle, idx, w, x, out)
-    est = time.perf_counter() - t0
-    while est * (args.steps + args.warmup) > 180 and sample > 8 * cfg.R:
-        sample = max(cfg.R, (sample // 2) - (sample // 2) % cfg.R)
-        idx, w, x, out = idx[:sample], w[:sample], x[:sample], out[:sample * cfg.K]
-        est /= 2
+    d = inputs.make_inputs(cfg, args.seed)
+    idx, w, x = d["topk_idx"], d["topk_weights"], d["x"]
+    out = inputs.make_out(cfg, cfg.T * cfg.K, args.seed)
+    lay = oracle.layout(idx, cfg.E, cfg.R)
     for _ in range(args.warmup):
-        cpu_oracle_step(oracle, idx, w, x, out)
+        oracle_step(oracle, cfg, idx, w, x, out)
     t0 = time.perf_counter()
     for _ in range(args.steps):
-        cpu_oracle_step(oracle, idx, w, x, out)
+        oracle_step(oracle, cfg, idx, w, x, out)
     el = time.perf_counter() - t0
-    value = sample * args.steps / el
-    desc = f"first {sample} tokens of {cfg.name} (all K picks, all R ranks), layout+dispatch+combine per step"
+    value = cfg.T * args.steps / el
+    desc = f"every step is one whole oracle step on the full {cfg.name} batch ({cfg.T} tokens), one thread"
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": el / args.steps * 1e3,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
-        "data": "synthetic", "config": {"workload": workload_text(cfg), "sample": desc},
+        "data": "synthetic", "config": config_object(cfg, max(1, args.gpus), lay.n_recv, lay.n_pairs),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
     print(json.dumps(line))
+
+
+# --------------------------------------------------------------------------- GPU measurement
+
+class Workload:
+    """Device buffers and the step of one configuration."""
+
+    def __init__(self, ep, inputs, cfg, rcfg, dev, seed, serial_layout=False):
+        self.ep, self.cfg, self.dev = ep, cfg, dev
+        T, K, H, E, R = cfg.T, cfg.K, cfg.H, cfg.E, cfg.R
+        d = inputs.make_inputs(rcfg, seed)
+        self.host = d
+        self.idx_h = torch.from_numpy(d["topk_idx"]).pin_memory()
+        self.w_h = torch.from_numpy(d["topk_weights"]).pin_memory()
+        self.x_h = torch.from_numpy(d["x"].view(np.int16)).view(torch.bfloat16).pin_memory()
+        self.idx, self.w, self.x = self.idx_h.to(dev), self.w_h.to(dev), self.x_h.to(dev)
+        self.out_h = inputs.make_out(rcfg, T * K, seed)              # expert outputs, pair space (seeded, host)
+        self.out = torch.from_numpy(self.out_h.view(np.int16)).view(torch.bfloat16).to(dev)
+        self.lay = ep.alloc_layout(T, K, E, R, device=dev)
+        self.ws = torch.empty(max(16, ep.ep_layout_workspace_bytes(T, K, E, R)), dtype=torch.uint8, device=dev)
+        self.ws2 = torch.empty_like(self.ws)
+        if cfg.host_staged:
+            self.recv = torch.empty(T * min(K, R), H, dtype=torch.bfloat16).pin_memory()
+        else:
+            self.recv = torch.empty(T * min(K, R), H, dtype=torch.bfloat16, device=dev)
+        self.y = torch.empty(T, H, dtype=torch.bfloat16, device=dev)
+        # big batches: the pair half of the layout runs beside dispatch; launch-bound batches keep one call
+        self.split_layout = (not serial_layout) and not is_small(cfg) and not cfg.host_staged
+        self.side = torch.cuda.Stream()
+        self.fork_ev, self.join_ev = torch.cuda.Event(), torch.cuda.Event()
+
+    def step(self, ev=None):
+        """layout -> dispatch -> combine. Dispatch needs only the receive-row half of the layout, so for big
+        batches the pair half (what combine needs) runs on a side stream while dispatch moves rows.
+        ev: optional dict of timing events recorded between the calls."""
+        ep, cfg, lay = self.ep, self.cfg, self.lay
+        E, R = cfg.E, cfg.R
+        main = torch.cuda.current_stream()
+        if ev:
+            ev["t0"].record()
+        if not self.split_layout:
+            ep.ep_layout(self.idx, E, R, out=lay, workspace=self.ws)
+        else:
+            self.fork_ev.record(main)                     # the side stream starts after everything queued so far
+            ep.ep_layout_ranks(self.idx, E, R, lay, self.ws)      # critical path first
+            self.side.wait_event(self.fork_ev)
+            if ev:
+                ev["p0"].record(self.side)
+            ep.ep_layout_pairs(self.idx, E, R, lay, self.ws2, stream=self.side)
+            if ev:
+                ev["p1"].record(self.side)
+            self.join_ev.record(self.side)
+        if ev:
+            ev["t1"].record()
+        ep.ep_dispatch(self.x, lay.recv_slot, self.recv, E, R, status=lay.status)
+        if ev:
+            ev["t2"].record()
+        if self.split_layout:
+            main.wait_event(self.join_ev)
+        if ev:
+            ev["t3"].record()
+        ep.ep_combine(self.out, lay.pair_slot, self.w, self.y, E, R, status=lay.status)
+        if ev:
+            ev["t4"].record()
+
+    @staticmethod
+    def new_events():
+        return {k: torch.cuda.Event(enable_timing=True) for k in ["t0", "t1", "t2", "t3", "t4", "p0", "p1"]}
+
+
+def measure(ep, wl, steps, warmup, rep, no_graph=False, sample_clocks=True):
+    """Times `steps` steps of a workload. Big workloads: back to back, direct launches, per-kernel events
+    inside the timed region. Small workloads: every step after an L2 flush, timed by its own event pair,
+    the step a CUDA-graph replay; per-kernel figures from a separate pass of direct launches."""
+    cfg, lay = wl.cfg, wl.lay
+    for _ in range(warmup):
+        wl.step()
+    torch.cuda.synchronize()
+    assert ep.ep_status(lay.status) == 0
+    n_recv, n_pairs = int(lay.rank_row_offsets[-1]), int(lay.expert_offsets[-1])
+    alg = algorithmic_bytes(cfg, n_recv, n_pairs)
+    small = is_small(cfg)
+    launches0 = ep.ep_launch_count()
+    dev_index = torch.cuda.current_device()
+    clocks = ClockSampler(dev_index) if sample_clocks else None
+    if not small:
+        evs = [wl.new_events() for _ in range(steps)]
+        start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        rep.barrier()
+        if clocks:
+            clocks.__enter__()
+        start.record()
+        for i in range(steps):
+            wl.step(evs[i])
+        stop.record()
+        torch.cuda.synchronize()
+        if clocks:
+            clocks.__exit__()
+        rep.barrier()
+        launches = ep.ep_launch_count() - launches0
+        total_ms = rep.max_over_ranks(start.elapsed_time(stop))
+        step_ms = [e["t0"].elapsed_time(e["t4"]) for e in evs]
+        launch_note = "direct launches"
+    else:
+        flusher = L2Flush(wl.dev)
+        graph = None
+        if not no_graph:
+            side = torch.cuda.Stream()
+            with torch.cuda.stream(side):
+                wl.step()
+            torch.cuda.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph):
+                wl.step()
+        s_ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+        e_ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+        rep.barrier()
+        if clocks:
+            clocks.__enter__()
+        for i in range(steps):
+            flusher()
+            s_ev[i].record()
+            graph.replay() if graph is not None else wl.step()
+            e_ev[i].record()
+        torch.cuda.synchronize()
+        if clocks:
+            clocks.__exit__()
+        rep.barrier()
+        launches = ep.ep_launch_count() - launches0
+        if graph is not None:          # replays launch the captured kernels without passing through the library
+            n0 = ep.ep_launch_count()
+            wl.step()
+            torch.cuda.synchronize()
+            launches = steps * (ep.ep_launch_count() - n0)
+        step_ms = [s.elapsed_time(e) for s, e in zip(s_ev, e_ev)]
+        total_ms = rep.max_over_ranks(sum(step_ms))
+        evs = [wl.new_events() for _ in range(min(steps, 50))]
+        for e in evs:                  # per-kernel figures: direct launches, each step after a flush
+            flusher()
+            wl.step(e)
+        torch.cuda.synchronize()
+        launch_note = "CUDA graph replay of one step" if graph is not None else "direct launches"
+        del flusher
+
+    def span(a, b):
+        return [e[a].elapsed_time(e[b]) for e in evs]
+
+    ops = {"layout": dict(stats_us(span("t0", "t1")),
+                          what="whole layout" if not wl.split_layout else "receive-row half (critical path)"),
+           "dispatch": dict(stats_us(span("t1", "t2")), bytes=alg["dispatch"]),
+           "combine": dict(stats_us(span("t3", "t4")), bytes=alg["combine"])}
+    if wl.split_layout:
+        ops["layout_pair_half"] = dict(stats_us(span("p0", "p1")), what="ep_layout_pairs on the side stream, beside dispatch")
+        ops["join_wait"] = dict(stats_us(span("t2", "t3")), what="main stream waiting for the pair half after dispatch")
+    for name in ("dispatch", "combine"):
+        o = ops[name]
+        o["GB/s"] = o["bytes"] / (o["us"] * 1e-6) / 1e9
+        o["best_GB/s"] = o["bytes"] / (o["best_us"] * 1e-6) / 1e9
+        o["tokens/s"] = cfg.T / (o["us"] * 1e-6)
+    if small:
+        ops["note"] = "per-kernel figures come from direct launches after a flush and include launch latency"
+    return {"total_ms": total_ms, "step": stats_us(step_ms), "ops": ops, "launches": int(launches),
+            "n_recv": n_recv, "n_pairs": n_pairs, "alg": alg, "launch": launch_note,
+            "layout": "one ep_layout call" if not wl.split_layout else
+            "ep_layout_ranks before dispatch, ep_layout_pairs on a side stream beside dispatch",
+            "clocks": clocks.summary() if clocks else None}
+
+
+def time_variants(ep, wl, n_recv, n_pairs, iters=20):
+    """Median device time of the variants around the path on the same batch: local grouping,
+    expanded dispatch, combine with per-rank partial outputs, dense all-gather / reduce-scatter."""
+    cfg, dev, lay = wl.cfg, wl.dev, wl.lay
+    T, K, H, E, R = cfg.T, cfg.K, cfg.H, cfg.E, cfg.R
+    row = 2 * H
+    flush = L2Flush(dev)
+    recv = torch.empty(max(1, n_recv), H, dtype=torch.bfloat16, device=dev)
+    ep.ep_dispatch(wl.x, lay.recv_slot, recv, E, R)
+    y = torch.empty(T, H, dtype=torch.bfloat16, device=dev)
+    res = {"rows": {"routed_receive": n_recv, "pairs": n_pairs, "dense": R * T}}
+
+    def timed(fn, nbytes):
+        ts = []
+        for _ in range(iters + 2):
+            flush()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            fn()
+            b.record()
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b))
+        ms = float(np.median(ts[2:]))
+        return {"us": ms * 1e3, "GB/s": nbytes / (ms * 1e-3) / 1e9, "bytes": nbytes}
+
+    grouped = torch.empty(max(1, n_pairs), H, dtype=torch.bfloat16, device=dev)
+    res["group (recv -> pair rows)"] = timed(lambda: ep.ep_group(recv, lay, grouped, E, R), 2 * row * n_pairs + 4 * n_pairs)
+    res["expanded dispatch (x -> pair rows)"] = timed(lambda: ep.ep_dispatch(wl.x, lay.pair_slot, grouped, E, R),
+                                                      row * T + row * n_pairs + 4 * T * K)
+    del grouped
+    partial = torch.empty(max(1, n_recv), H, dtype=torch.bfloat16, device=dev)
+    res["combine with partial outputs (2 kernels)"] = timed(
+        lambda: ep.ep_combine_partial(wl.out, lay, wl.w, partial, y, E, R),
+        row * n_pairs + 2 * row * n_recv + row * T + 16 * T * K)
+    del partial
+    gathered = torch.empty(R * T, H, dtype=torch.bfloat16, device=dev)
+    res["dense all-gather"] = timed(lambda: ep.ep_dense_allgather(wl.x, gathered, K, E, R), row * T + row * R * T)
+    if R <= 32:
+        res["dense reduce-scatter (2 kernels)"] = timed(
+            lambda: ep.ep_dense_reduce_scatter(wl.idx, wl.out, lay.pair_slot, wl.w, gathered, y, E, R),
+            row * n_pairs + 2 * row * R * T + row * T + 12 * T * K)
+    del gathered, flush
+    return res
+
+
+def host_staged_arms(ep, wl, iters=10, sweep=True):
+    """Receive buffer in mapped pinned host memory: (i) the dispatch kernel stores straight
+    into it; (ii) dispatch packs into device staging and the copy engine moves each rank's
+    partition; plus the host-link probe both are measured against, and the round trips."""
+    cfg, dev, lay, x, recv_host = wl.cfg, wl.dev, wl.lay, wl.x, wl.recv
+    E, R = cfg.E, cfg.R
+    n_recv = int(lay.rank_row_offsets[-1])
+    row = 2 * cfg.H
+    staging = torch.empty(recv_host.shape[0], cfg.H, dtype=torch.bfloat16, device=dev)
+    probe_src = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    probe_dst = torch.empty(256 << 20, dtype=torch.uint8).pin_memory()
+    d2h = ep.ep_probe_bandwidth(ep.PROBE_MEMCPY, probe_dst, probe_src, 256 << 20, iters=10)
+    h2d = ep.ep_probe_bandwidth(ep.PROBE_MEMCPY, probe_src, probe_dst, 256 << 20, iters=10)
+    del probe_src, probe_dst
+
+    def timed(fn):
+        best = 1e30
+        for _ in range(iters + 1):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            fn()
+            b.record()
+            torch.cuda.synchronize()
+            best = min(best, a.elapsed_time(b))
+        return best
+
+    def arm_kernel():
+        ep.ep_dispatch(x, lay.recv_slot, recv_host, E, R)
+
+    offs_pinned = torch.zeros(R + 1, dtype=torch.int32).pin_memory()
+
+    def arm_copy_known():           # the offsets first travel to the host: one small copy and a stream sync, timed
+        offs_pinned.copy_(lay.rank_row_offsets, non_blocking=True)
+        torch.cuda.current_stream().synchronize()
+        ep.ep_dispatch_copy_engine(x, lay.recv_slot, staging, recv_host, E, R, rank_row_offsets_host=offs_pinned)
+
+    def arm_copy_blind():           # no count reaches the host: one copy of the worst-case T*min(K,R) rows
+        ep.ep_dispatch_copy_engine(x, lay.recv_slot, staging, recv_host, E, R, rank_row_offsets_host=None)
+
+    res = {"host_link_d2h_GB/s": d2h, "host_link_h2d_GB/s": h2d, "rows": n_recv, "bytes_over_link": n_recv * row}
+    for name, fn, nbytes in [("kernel_store", arm_kernel, n_recv * row),
+                             ("copy_engine_per_rank", arm_copy_known, n_recv * row),
+                             ("copy_engine_worst_case", arm_copy_blind, recv_host.shape[0] * row)]:
+        ms = timed(fn)
+        res[name] = {"us": ms * 1e3, "GB/s": nbytes / (ms * 1e-3) / 1e9, "useful_GB/s": n_recv * row / (ms * 1e-3) / 1e9,
+                     "frac_of_d2h_probe": n_recv * row / (ms * 1e-3) / 1e9 / d2h, "tokens/s": cfg.T / (ms * 1e-3)}
+    # dispatch round trip through the bounce buffer on two streams: all uploads then all downloads, or chunk-wise duplex
+    cap = recv_host.shape[0]
+    bounce = torch.empty(2 * cap, cfg.H, dtype=torch.bfloat16).pin_memory()
+    back = torch.empty(cap, cfg.H, dtype=torch.bfloat16, device=dev)
+    up, down = torch.cuda.Stream(), torch.cuda.Stream()
+    offs_host = lay.rank_row_offsets.cpu()
+    torch.cuda.synchronize()
+    trips = {}
+    for duplex, chunks in ([(0, 1), (1, 1), (1, 2), (1, 4), (1, 8)] if sweep else [(0, 1), (1, 1)]):
+        best = 1e30
+        for rnd in range(iters + 1):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(down)
+            ep.ep_host_roundtrip(x, lay.recv_slot, offs_host, staging, bounce, back, E, R, round=rnd,
+                                 chunks_per_rank=chunks, duplex=bool(duplex), stream_up=up, stream_down=down)
+            b.record(down)
+            torch.cuda.synchronize()
+            best = min(best, a.elapsed_time(b))
+        trips[("duplex" if duplex else "serial") + f", {chunks} chunk(s) per rank"] = {
+            "us": best * 1e3, "GB/s_each_way": n_recv * row / (best * 1e-3) / 1e9, "tokens/s": cfg.T / (best * 1e-3)}
+    res["roundtrip"] = trips
+    # cost of one completion check: the wait kernel on flags that are already posted
+    n_s = max(1, R - 1)
+    flags_dev = torch.full((64,), 3, dtype=torch.int32, device=dev)
+    flags_pin = torch.full((64,), 3, dtype=torch.int32).pin_memory()
+    waits = {}
+    for name, fl in [("flags in device memory", flags_dev), ("flags in pinned host memory", flags_pin)]:
+        waits[name] = {"us": timed(lambda: ep.ep_wait_senders(fl, n_s, 3, 100_000_000)) * 1e3, "senders": n_s}
+    res["flag_wait_posted"] = waits
+    return res
+
+
+def roofline_object(cfg, name, achieved, peak, peak_kind, probes=None):
+    r = {"bound": "hbm", "kernel": name, "achieved": achieved, "peak": peak, "peak_kind": peak_kind + " copy peak",
+         "unit": "GB/s", "frac": achieved / peak, "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS,
+         "traffic": NCU_TRAFFIC_BYTES.get((cfg.name, name))}
+    if probes:
+        r["frac_of_own_copy_probe"] = achieved / probes["copy_GB/s"]
+    return r
+
+
+def summarize_config(cfg, m, peak, host=None):
+    """The entry of one extra configuration under `configs`."""
+    ops = m["ops"]
+    e = {"workload": workload_text(cfg), "step": m["step"], "tokens/s": cfg.T / (m["step"]["us"] * 1e-6),
+         "launch": m["launch"], "layout_call": m["layout"], "n_recv": m["n_recv"], "n_pairs": m["n_pairs"], "ops": ops}
+    for name in ("dispatch", "combine"):
+        ops[name]["frac_of_measured_peak"] = ops[name]["GB/s"] / peak
+        ops[name]["frac_of_nominal_8000"] = ops[name]["GB/s"] / NOMINAL_HBM_GBS
+    if step_bytes_estimate(cfg) < L2_BYTES:
+        e["note"] = "launch-latency-bound: the whole step moves less than L2 holds; HBM fractions are not meaningful"
+    if host is not None:
+        link = host["host_link_d2h_GB/s"]
+        e["host_link"] = {"bound": "host-link", "peak": link, "peak_kind": "cudaMemcpyAsync D2H probe, 256 MB pinned, same run",
+                          "unit": "GB/s", "kernel_store": {"achieved": host["kernel_store"]["useful_GB/s"],
+                                                           "frac": host["kernel_store"]["frac_of_d2h_probe"]},
+                          "copy_engine_per_rank": {"achieved": host["copy_engine_per_rank"]["useful_GB/s"],
+                                                   "frac": host["copy_engine_per_rank"]["frac_of_d2h_probe"]}}
+        e["host_staged"] = host
+    return e
 
 
 def main():
@@ -346,6 +588,8 @@ def main():
                     help="one ep_layout call instead of the receive-row half before dispatch and the pair half beside it")
     ap.add_argument("--variants", action="store_true",
                     help="also time the variants around the path (grouping, partial-output combine, dense baseline)")
+    ap.add_argument("--no-configs", action="store_true", help="skip the extra configurations under `configs`")
+    ap.add_argument("--config-steps", type=int, default=50, help="timed steps of each extra configuration")
     ap.add_argument("--seed", type=int, default=0)
     args = ap.parse_args()
     if args.warmup < 3:
@@ -369,128 +613,13 @@ def main():
     rcfg = inputs.shard_config(cfg, rank)            # replica `rank`: same shapes, its own seed stream
     T, K, H, E, R = cfg.T, cfg.K, cfg.H, cfg.E, cfg.R
 
-    # ---- inputs (seeded; the routing, weights and activations come from the host generators)
-    d = inputs.make_inputs(rcfg, args.seed)
-    idx_h = torch.from_numpy(d["topk_idx"]).pin_memory()
-    w_h = torch.from_numpy(d["topk_weights"]).pin_memory()
-    x_h = torch.from_numpy(d["x"].view(np.int16)).view(torch.bfloat16).pin_memory()
-    idx, w, x = idx_h.to(dev), w_h.to(dev), x_h.to(dev)
-    out_h = inputs.make_out(rcfg, T * K, args.seed)                   # expert outputs, pair space (seeded, host)
-    out = torch.from_numpy(out_h.view(np.int16)).view(torch.bfloat16).to(dev)
-    lay = ep.alloc_layout(T, K, E, R, device=dev)
-    ws = torch.empty(max(16, ep.ep_layout_workspace_bytes(T, K, E, R)), dtype=torch.uint8, device=dev)
-    recv = torch.empty(T * min(K, R), H, dtype=torch.bfloat16, device=dev)
-    y = torch.empty(T, H, dtype=torch.bfloat16, device=dev)
-    if cfg.host_staged:
-        recv = torch.empty(T * min(K, R), H, dtype=torch.bfloat16).pin_memory()
+    wl = Workload(ep, inputs, cfg, rcfg, dev, args.seed, serial_layout=args.serial_layout)
+    m = measure(ep, wl, args.steps, args.warmup, rep, no_graph=args.no_graph)
+    n_recv, n_pairs, alg = m["n_recv"], m["n_pairs"], m["alg"]
+    value = world * T * args.steps / (m["total_ms"] * 1e-3)
 
-    # big batches: the pair half of the layout runs beside dispatch; launch-bound batches keep one call
-    est_bytes = 2 * H * (2 * T + T * min(K, R) + T * K)
-    split_layout = (not args.serial_layout) and est_bytes >= 4 * L2_BYTES and not cfg.host_staged
-    ws2 = torch.empty_like(ws)
-    side = torch.cuda.Stream()
-    fork_ev, join_ev = torch.cuda.Event(), torch.cuda.Event()
-
-    def step(events=None):
-        """layout -> dispatch -> combine. Dispatch needs only the receive-row half of the layout, so the
-        pair half (what combine needs) runs on a side stream while dispatch moves rows."""
-        main = torch.cuda.current_stream()
-        if events:
-            events[0].record()
-        if not split_layout:
-            ep.ep_layout(idx, E, R, out=lay, workspace=ws)
-        else:
-            fork_ev.record(main)                      # the side stream starts after everything queued so far
-            ep.ep_layout_ranks(idx, E, R, lay, ws)    # critical path first
-            side.wait_event(fork_ev)
-            ep.ep_layout_pairs(idx, E, R, lay, ws2, stream=side)
-            join_ev.record(side)
-        if events:
-            events[1].record()
-        ep.ep_dispatch(x, lay.recv_slot, recv, E, R, status=lay.status)
-        if split_layout:
-            main.wait_event(join_ev)
-        if events:
-            events[2].record()
-        ep.ep_combine(out, lay.pair_slot, w, y, E, R, status=lay.status)
-        if events:
-            events[3].record()
-
-    for _ in range(args.warmup):
-        step()
-    torch.cuda.synchronize()
-    assert ep.ep_status(lay.status) == 0
-    n_recv, n_pairs = int(lay.rank_row_offsets[-1]), int(lay.expert_offsets[-1])
-    alg = algorithmic_bytes(cfg, n_recv, n_pairs)
-    step_bytes = alg["dispatch"] + alg["combine"]
-    small = step_bytes < 4 * L2_BYTES and not cfg.host_staged       # the step's data could (partly) stay in L2
-
-    launches0 = ep.ep_launch_count()
-    if not small:
-        # ---- timed region: K steps back to back, device-timed, per-kernel events on the launching stream
-        evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
-        start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        rep.barrier()
-        with ClockSampler(torch.cuda.current_device()) as clocks:
-            start.record()
-            for i in range(args.steps):
-                step(evs[i])
-            stop.record()
-            torch.cuda.synchronize()
-        rep.barrier()
-        launches = ep.ep_launch_count() - launches0
-        total_ms = rep.max_over_ranks(start.elapsed_time(stop))
-        per = np.array([[e[j].elapsed_time(e[j + 1]) for j in range(3)] for e in evs])  # ms: layout, dispatch, combine
-        l2_note = "working set per step exceeds L2 several times over (no flush needed)"
-        launch_note = "direct launches"
-    else:
-        # ---- small workloads: L2 is flushed (256 MB written) before every step; each step is timed by its own
-        # event pair and the step itself is a CUDA-graph replay, so host launch cost is not what is measured
-        flusher = L2Flush(dev)
-        graph = None
-        if not args.no_graph:
-            side = torch.cuda.Stream()
-            with torch.cuda.stream(side):
-                step()
-            torch.cuda.synchronize()
-            graph = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(graph):
-                step()
-        s_ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
-        e_ev = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps)]
-        rep.barrier()
-        with ClockSampler(torch.cuda.current_device()) as clocks:
-            for i in range(args.steps):
-                flusher()
-                s_ev[i].record()
-                graph.replay() if graph is not None else step()
-                e_ev[i].record()
-            torch.cuda.synchronize()
-        rep.barrier()
-        launches = ep.ep_launch_count() - launches0
-        if graph is not None:                   # replays launch the captured kernels without passing through the library
-            launches = args.steps * launches_per_step(ep, step)
-        total_ms = rep.max_over_ranks(sum(s.elapsed_time(e) for s, e in zip(s_ev, e_ev)))
-        # per-kernel figures from a separate pass of direct launches, each step after a flush
-        evs = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(min(args.steps, 50))]
-        for e in evs:
-            flusher()
-            step(e)
-        torch.cuda.synchronize()
-        per = np.array([[e[j].elapsed_time(e[j + 1]) for j in range(3)] for e in evs])
-        l2_note = ("step data would fit L2: before every timed step 256 MB are written and then another 256 MB read "
-                   "(L2 left holding clean foreign lines); each step timed by its own event pair")
-        launch_note = "CUDA graph replay of one step" if graph is not None else "direct launches"
-        del flusher
-    lay_ms, dis_ms, com_ms = [float(v) for v in per.mean(axis=0)]
-    value = world * T * args.steps / (total_ms * 1e-3)
-
-    # ---- host-staged variant: the two arms of the receive path and the host-link probe
-    host = None
-    if cfg.host_staged:
-        host = host_staged_arms(ep, cfg, x, lay, recv, dev)
-
-    variants = time_variants(ep, cfg, idx, w, x, out, lay, n_recv, n_pairs, dev) if args.variants else None
+    host = host_staged_arms(ep, wl) if cfg.host_staged else None
+    variants = time_variants(ep, wl, n_recv, n_pairs) if args.variants else None
 
     # ---- end to end: one C-ABI call per step, host buffers in, host buffer out
     arena = torch.empty(ep.ep_host_step_arena_bytes(T, K, H, E, R), dtype=torch.uint8, device=dev)
@@ -501,7 +630,8 @@ def main():
     s_in, s_comp, s_out = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()
 
     def e2e_step():
-        ep.ep_host_step_pipelined(x_h, idx_h, w_h, y_h, arena, E, R, e2e_chunks, s_in, s_comp, s_out, status_host=st_h)
+        ep.ep_host_step_pipelined(wl.x_h, wl.idx_h, wl.w_h, y_h, arena, E, R, e2e_chunks, s_in, s_comp, s_out,
+                                  status_host=st_h)
 
     torch.cuda.synchronize()
     for _ in range(3 if args.e2e_steps > 0 else 0):
@@ -517,7 +647,7 @@ def main():
     e2e_ms = rep.max_over_ranks(e0.elapsed_time(e1))
     assert int(st_h[0]) == 0
     e2e_value = world * T * args.e2e_steps / (e2e_ms * 1e-3) if args.e2e_steps > 0 else None
-    h2d = x_h.numel() * 2 + idx_h.numel() * 4 + w_h.numel() * 4
+    h2d = wl.x_h.numel() * 2 + wl.idx_h.numel() * 4 + wl.w_h.numel() * 4
     d2h = y_h.numel() * 2 + 4
     del arena
 
@@ -532,45 +662,45 @@ def main():
         probes["what"] = "ep_probe_bandwidth, 1 GiB, best of 8; copy counts read + write bytes"
         del pa, pb
 
+    peak, peak_kind = measured_peak()
+
+    # ---- the other configurations, same protocol, fewer steps (one GPU only: they are not part of `value`)
+    configs = None
+    if world == 1 and not args.no_configs:
+        configs = {}
+        for name in ["C1", "C2", "C3", "C5"]:
+            if name == cfg.name:
+                continue
+            c = inputs.CONFIGS[name]
+            w2 = Workload(ep, inputs, c, c, dev, args.seed)
+            m2 = measure(ep, w2, args.config_steps, max(5, args.warmup), rep, sample_clocks=False)
+            h2 = host_staged_arms(ep, w2, iters=6, sweep=False) if c.host_staged else None
+            configs[name] = summarize_config(c, m2, peak, h2)
+            del w2
+            torch.cuda.empty_cache()
+
     if rank != 0:
         rep.close()
         return
-    peak, peak_kind = measured_peak()
-    com_gbs = alg["combine"] / (com_ms * 1e-3) / 1e9
-    dis_gbs = alg["dispatch"] / (dis_ms * 1e-3) / 1e9
-
-    def roof(achieved, name):
-        r = {"bound": "hbm", "kernel": name, "achieved": achieved, "peak": peak, "peak_kind": peak_kind + " copy peak",
-             "unit": "GB/s", "frac": achieved / peak, "frac_of_nominal_8000": achieved / NOMINAL_HBM_GBS,
-             "traffic": NCU_TRAFFIC_BYTES.get((cfg.name, name))}
-        if probes:
-            r["frac_of_own_copy_probe"] = achieved / probes["copy_GB/s"]
-        return r
-
+    ops = m["ops"]
+    com_gbs, dis_gbs = ops["combine"]["GB/s"], ops["dispatch"]["GB/s"]
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": args.warmup, "ms_per_step": total_ms / args.steps, "higher_is_better": True,
+        "warmup": args.warmup, "ms_per_step": m["total_ms"] / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": workload_text(cfg), "parallelism": f"{world} independent replica(s)",
-                   "l2": l2_note, "launch": launch_note, "n_recv": n_recv, "n_pairs": n_pairs,
-                   "layout": "one ep_layout call" if not split_layout else
-                   "ep_layout_ranks before dispatch, ep_layout_pairs on a side stream beside dispatch"},
-        "ops": {
-            "layout": {"us": lay_ms * 1e3, "what": "whole layout" if not split_layout else "receive-row half (critical path)"},
-            "dispatch": {"us": dis_ms * 1e3, "GB/s": dis_gbs, "tokens/s": T / (dis_ms * 1e-3), "bytes": alg["dispatch"]},
-            "combine": {"us": com_ms * 1e3, "GB/s": com_gbs, "tokens/s": T / (com_ms * 1e-3), "bytes": alg["combine"]},
-        },
-        "roofline": roof(com_gbs, "combine_rows_kernel"),
-        "roofline_dispatch": roof(dis_gbs, "dispatch_rows_kernel"),
+        "config": config_object(cfg, world, n_recv, n_pairs),
+        "protocol": {"launch": m["launch"], "layout": m["layout"], "step": m["step"]},
+        "ops": ops,
+        "roofline": roofline_object(cfg, "combine_rows_kernel", com_gbs, peak, peak_kind, probes),
+        "roofline_dispatch": roofline_object(cfg, "dispatch_rows_kernel", dis_gbs, peak, peak_kind, probes),
         "probes": probes,
-        "clocks": clocks.summary(),
+        "clocks": m["clocks"],
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": e2e_ms / n_e2e, "steps": args.e2e_steps,
                 "call": f"ep_host_step_pipelined (layout+dispatch+group+combine, pinned host in/out, {e2e_chunks} token "
                         "chunk(s) on upload/compute/download streams)"},
-        "gpu_launches": int(launches),
-        "context": "paper reports 2.00x (dispatch) / 1.53x (combine) over NCCL for its dense all-gather/"
-                   "reduce-scatter on RTX 4090/5090 PCIe boxes; no number for the routing-aware path",
+        "gpu_launches": m["launches"],
+        "context": CONTEXT,
     }
     if variants is not None:
         line["variants"] = variants
@@ -581,11 +711,11 @@ def main():
                                      "achieved": host["kernel_store"]["GB/s"], "peak": link,
                                      "peak_kind": "cudaMemcpyAsync D2H probe, 256 MB pinned, same run", "unit": "GB/s",
                                      "frac": host["kernel_store"]["GB/s"] / link, "traffic": None}
+    if configs is not None:
+        line["configs"] = configs
     if not args.no_cpu_baseline:
-        v, n, el = time_oracle(cfg, d["topk_idx"], d["topk_weights"], d["x"], out_h, min_seconds=10.0, max_steps=20)
-        line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle",
-                                "sample": f"{n} whole step(s) of the same {cfg.name} batch in {el:.1f} s, one thread",
-                                "host_cores_available": os.cpu_count()}
+        line["cpu_baseline"] = time_oracle(cfg, wl.host["topk_idx"], wl.host["topk_weights"], wl.host["x"], wl.out_h,
+                                           min_seconds=8.0, max_steps=20)
     print(json.dumps(line))
     rep.close()
 

@@ -95,6 +95,29 @@ def dispatch(x_bits: np.ndarray, recv_slot: np.ndarray, recv_rows: int, fill: in
     return recv
 
 
+def dispatch_into(x_bits: np.ndarray, recv_slot: np.ndarray, recv: np.ndarray) -> None:
+    """`dispatch` for a contiguous range of tokens into a receive buffer the caller owns (the
+    benchmark's all-cores leg calls it once per token range; the C function is the same)."""
+    assert x_bits.flags.c_contiguous and recv_slot.flags.c_contiguous and recv.flags.c_contiguous
+    assert x_bits.dtype == np.uint16 and recv_slot.dtype == np.int32 and recv.dtype == np.uint16
+    T, H = x_bits.shape
+    rc = _load().ep_oracle_dispatch(T, recv_slot.shape[1], H, _p(x_bits), _p(recv_slot), _p(recv),
+                                    ctypes.c_int64(recv.shape[0]))
+    if rc != 0:
+        raise ValueError("oracle dispatch: slot beyond recv_rows")
+
+
+def combine_f32_into(out_bits: np.ndarray, slot: np.ndarray, w: np.ndarray, y: np.ndarray) -> None:
+    """`combine_f32` for a contiguous range of tokens into rows of `y` the caller owns."""
+    assert out_bits.flags.c_contiguous and slot.flags.c_contiguous and w.flags.c_contiguous and y.flags.c_contiguous
+    assert out_bits.dtype == np.uint16 and slot.dtype == np.int32 and w.dtype == np.float32 and y.dtype == np.uint16
+    T, K = slot.shape
+    rc = _load().ep_oracle_combine_f32(T, K, out_bits.shape[1], _p(out_bits), ctypes.c_int64(out_bits.shape[0]),
+                                       _p(slot), _p(w), _p(y))
+    if rc != 0:
+        raise ValueError("oracle combine: slot beyond out rows")
+
+
 def combine_f32(out_bits: np.ndarray, slot: np.ndarray, w: np.ndarray) -> np.ndarray:
     out = np.ascontiguousarray(out_bits, dtype=np.uint16)
     s = np.ascontiguousarray(slot, dtype=np.int32)

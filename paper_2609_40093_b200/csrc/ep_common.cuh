@@ -6,6 +6,8 @@
 #include <cuda_bf16.h>
 #include <stdint.h>
 
+#include <mutex>
+
 #include "../../include/ep.h"
 
 namespace ep {
@@ -19,6 +21,12 @@ constexpr unsigned kFullMask = 0xffffffffu;
 
 void note_cuda_error(cudaError_t e);       // remembers the code for ep_last_cuda_error
 void count_launches(int n);                // feeds ep_launch_count
+
+// Ordering events of the multi-stream entry points: *pool gets at least `need` timing-free events of
+// the current device; `hold` owns the pool's mutex until the caller lets go of it (after its last
+// record/wait has been enqueued). At most kOrderEventPool events per call.
+constexpr int kOrderEventPool = 1024;
+int order_events(cudaEvent_t **pool, int need, std::unique_lock<std::mutex> &hold);
 
 #define EP_CUDA_TRY(expr)                                   \
     do {                                                    \
@@ -35,6 +43,22 @@ void count_launches(int n);                // feeds ep_launch_count
         ::ep::count_launches(n_launched);                   \
         EP_CUDA_TRY(cudaGetLastError());                    \
     } while (0)
+
+// Kernel launchers shared between the translation units (arguments already validated).
+int launch_dispatch(const ep_shape_t &s, const void *x, const int32_t *recv_slot, void *recv,
+                    int64_t capacity_rows, int32_t *status, cudaStream_t stream);
+int launch_group(const ep_shape_t &s, const void *recv, int64_t recv_rows, const int32_t *pair_row,
+                 const int32_t *n_pairs, void *grouped, int64_t capacity_rows, int32_t *status,
+                 cudaStream_t stream);
+int launch_combine(const ep_shape_t &s, const void *out, int64_t out_rows, const int32_t *slot,
+                   const float *weights, void *y, int32_t *status, cudaStream_t stream);
+int launch_permute(int hidden, const void *src, int64_t src_rows, const int32_t *src_slot, void *dst,
+                   int64_t dst_rows, const int32_t *dst_slot, int64_t n, int32_t *status, cudaStream_t stream);
+int launch_partial_rows(const ep_shape_t &s, const void *out, int64_t out_rows, const int32_t *pair_slot,
+                        const int32_t *recv_slot, const float *weights, void *partial, int64_t partial_rows,
+                        int32_t *status, cudaStream_t stream);
+int launch_sum_partial_rows(int hidden, int top_k, const void *partial, int64_t partial_rows, const int32_t *slot,
+                            void *y, int n_tokens, int32_t *status, cudaStream_t stream);
 
 inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 

@@ -8,36 +8,29 @@
 
 namespace ep {
 
-int launch_dispatch(const ep_shape_t &s, const void *x, const int32_t *recv_slot, void *recv,
-                    int64_t capacity_rows, int32_t *status, cudaStream_t stream);
-int launch_group(const ep_shape_t &s, const void *recv, int64_t recv_rows, const int32_t *pair_row,
-                 const int32_t *n_pairs, void *grouped, int64_t capacity_rows, int32_t *status,
-                 cudaStream_t stream);
-int launch_combine(const ep_shape_t &s, const void *out, int64_t out_rows, const int32_t *slot,
-                   const float *weights, void *y, int32_t *status, cudaStream_t stream);
-int launch_permute(int hidden, const void *src, int64_t src_rows, const int32_t *src_slot, void *dst,
-                   int64_t dst_rows, const int32_t *dst_slot, int64_t n, int32_t *status, cudaStream_t stream);
-
 namespace {
 std::atomic<int> g_last_cuda_error{0};
 std::atomic<long long> g_launches{0};
 }  // namespace
 
-// Timing-free events for cross-stream ordering: created on first use, kept for the life of the process.
+// Timing-free events for cross-stream ordering: created on first use, kept for the life of the
+// process (events hold no device memory). One pool per device, shared by every multi-stream entry
+// point; `hold` keeps the pool's mutex until the caller has enqueued its whole sequence, so that
+// two host threads cannot interleave their records and waits on the same events. (A wait that has
+// been enqueued keeps the state the event had then; a later record by another call does not move it.)
 namespace {
-constexpr int kEventPool = 1024;
-cudaEvent_t g_events[64][kEventPool];
+cudaEvent_t g_events[64][kOrderEventPool];
 int g_events_ready[64] = {};
 std::mutex g_event_mutex;
 }  // namespace
 
-int order_events(cudaEvent_t **pool, int need)
+int order_events(cudaEvent_t **pool, int need, std::unique_lock<std::mutex> &hold)
 {
-    if (need > kEventPool) return EP_ERR_INVALID_ARG;
+    if (need > kOrderEventPool) return EP_ERR_INVALID_ARG;
     int dev = 0;
     EP_CUDA_TRY(cudaGetDevice(&dev));
     if (dev < 0 || dev >= 64) return EP_ERR_INVALID_ARG;
-    std::lock_guard<std::mutex> lock(g_event_mutex);
+    hold = std::unique_lock<std::mutex>(g_event_mutex);
     while (g_events_ready[dev] < need) {
         EP_CUDA_TRY(cudaEventCreateWithFlags(&g_events[dev][g_events_ready[dev]], cudaEventDisableTiming));
         ++g_events_ready[dev];
@@ -243,7 +236,8 @@ extern "C" int ep_host_step_pipelined(const ep_shape_t *shape, const void *x_hos
     cudaStream_t in = static_cast<cudaStream_t>(stream_in_), comp = static_cast<cudaStream_t>(stream_compute_),
                  outs = static_cast<cudaStream_t>(stream_out_);
     cudaEvent_t *ev = nullptr;
-    rc = order_events(&ev, 2 * chunks + 3);
+    std::unique_lock<std::mutex> hold;
+    rc = order_events(&ev, 2 * chunks + 3, hold);
     if (rc != EP_OK) return rc;
     const size_t T = shape->num_tokens, K = shape->top_k, H = shape->hidden;
     // the arena is reused from step to step: uploads wait for the previous step's kernels, and the

@@ -85,7 +85,9 @@ LayoutPlan make_plan(const ep_shape_t &s)
         p.mode = p.n_ctas <= kMaxCluster ? kModeCluster : kModeGlobal;
     }
     p.smem = pw * p.warps + pc;
-    p.workspace_bytes = p.mode == kModeGlobal ? sizeof(int32_t) * (size_t)p.n_ctas * p.bins : 16;
+    // the cluster form needs no scratch, but falls back to the global form on a device that cannot
+    // keep the whole cluster resident, so both ask for cta_part
+    p.workspace_bytes = p.mode == kModeSingle ? 16 : sizeof(int32_t) * (size_t)p.n_ctas * p.bins;
     return p;
 }
 
@@ -395,6 +397,32 @@ extern "C" size_t ep_layout_workspace_bytes(const ep_shape_t *shape)
 namespace ep {
 namespace {
 
+// Can `cfg` (one cluster = the whole grid) be resident on device `dev`? Asked once per device and
+// (cluster size, CTA size, shared memory) and remembered; "no" sends the call to the global form.
+bool cluster_fits(int dev, const cudaLaunchConfig_t &cfg)
+{
+    struct Key {
+        int dev;
+        unsigned ctas, threads;
+        size_t smem;
+        bool fits;
+    };
+    static std::mutex mu;
+    static Key known[32];
+    static int n_known = 0;
+    std::lock_guard<std::mutex> lock(mu);
+    for (int i = 0; i < n_known; ++i)
+        if (known[i].dev == dev && known[i].ctas == cfg.gridDim.x && known[i].threads == cfg.blockDim.x &&
+            known[i].smem == cfg.dynamicSmemBytes)
+            return known[i].fits;
+    int n = 0;
+    const cudaError_t e = cudaOccupancyMaxActiveClusters(&n, layout_assign_kernel, &cfg);
+    if (e != cudaSuccess) (void)cudaGetLastError();         // treated as "does not fit"; not this call's error
+    const bool fits = e == cudaSuccess && n >= 1;
+    if (n_known < 32) known[n_known++] = Key{dev, cfg.gridDim.x, cfg.blockDim.x, cfg.dynamicSmemBytes, fits};
+    return fits;
+}
+
 int run_layout(const ep_shape_t *shape, const int32_t *topk_idx, const ep_layout_t *out, void *workspace,
                size_t workspace_bytes, void *stream_, int parts)
 {
@@ -460,7 +488,13 @@ int run_layout(const ep_shape_t *shape, const int32_t *topk_idx, const ep_layout
         attr.val.clusterDim.z = 1;
         cfg.attrs = &attr;
         cfg.numAttrs = 1;
-    } else if (plan.mode == kModeGlobal) {
+        if (!cluster_fits(dev, cfg)) {                      // this device cannot co-schedule the cluster
+            a.mode = kModeGlobal;
+            cfg.attrs = nullptr;
+            cfg.numAttrs = 0;
+        }
+    }
+    if (a.mode == kModeGlobal) {
         layout_cta_count_kernel<<<plan.n_ctas, plan.warps * 32, plan.smem, stream>>>(a);
         // the main kernel may start while the first still runs; it waits on the device before it reads cta_part
         attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;

@@ -13,9 +13,6 @@
 
 namespace ep {
 
-int launch_dispatch(const ep_shape_t &s, const void *x, const int32_t *recv_slot, void *recv,
-                    int64_t capacity_rows, int32_t *status, cudaStream_t stream);
-int order_events(cudaEvent_t **pool, int need);
 
 namespace {
 
@@ -115,7 +112,8 @@ extern "C" int ep_host_roundtrip(const ep_shape_t *shape, const void *x, const i
         if (rank_row_offsets_host[r + 1] < rank_row_offsets_host[r]) return EP_ERR_INVALID_ARG;
     cudaStream_t up = static_cast<cudaStream_t>(stream_up_), down = static_cast<cudaStream_t>(stream_down_);
     cudaEvent_t *ev = nullptr;
-    rc = order_events(&ev, R * chunks_per_rank + 2);
+    std::unique_lock<std::mutex> hold;
+    rc = order_events(&ev, R * chunks_per_rank + 2, hold);
     if (rc != EP_OK) return rc;
     const size_t row_bytes = (size_t)shape->hidden * 2;
     // two bounce buffers alternate by round, so a buffer is reused only every other round

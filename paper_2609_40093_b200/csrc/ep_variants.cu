@@ -244,6 +244,35 @@ dense_allgather_kernel(const uint4 *__restrict__ x, uint4 *gathered, int T, int 
 }
 
 }  // namespace
+
+// Stage 1 of the routed two-stage combine: partial[recv_slot[t][k]] = bf16(fma chain of the k's sharing that row).
+int launch_partial_rows(const ep_shape_t &s, const void *out, int64_t out_rows, const int32_t *pair_slot,
+                        const int32_t *recv_slot, const float *weights, void *partial, int64_t partial_rows,
+                        int32_t *status, cudaStream_t stream)
+{
+    const int T = s.num_tokens, vpr = s.hidden / 8;
+    const GroupPlan p = plan_group(vpr);
+    reduce_to_rows_kernel<<<ceil_div(T, p.rows_per_block), p.block, 0, stream>>>(
+        static_cast<const uint4 *>(out), out_rows, pair_slot, recv_slot, nullptr, weights, static_cast<uint4 *>(partial),
+        partial_rows, T, s.top_k, s.num_experts, s.num_ranks, vpr, p.G, status);
+    EP_LAUNCH_CHECK(1);
+    return EP_OK;
+}
+
+// Stage 2 for `n_tokens` tokens starting at the rows the pointers name: y[t] = bf16(sum of the token's
+// distinct partial rows in the order of their first k). slot and y point at the first token of the range.
+int launch_sum_partial_rows(int hidden, int top_k, const void *partial, int64_t partial_rows, const int32_t *slot,
+                            void *y, int n_tokens, int32_t *status, cudaStream_t stream)
+{
+    if (n_tokens <= 0) return EP_OK;
+    const int vpr = hidden / 8;
+    const GroupPlan p = plan_group(vpr);
+    sum_rows_kernel<<<ceil_div(n_tokens, p.rows_per_block), p.block, 0, stream>>>(
+        static_cast<const uint4 *>(partial), partial_rows, slot, static_cast<uint4 *>(y), n_tokens, top_k, vpr, p.G, status);
+    EP_LAUNCH_CHECK(1);
+    return EP_OK;
+}
+
 }  // namespace ep
 
 extern "C" int ep_combine_partial(const ep_shape_t *shape, const void *out, int64_t out_rows,
@@ -259,17 +288,11 @@ extern "C" int ep_combine_partial(const ep_shape_t *shape, const void *out, int6
     if (!aligned16(out) || !aligned16(partial) || !aligned16(y) || out_rows < 0 || partial_capacity_rows < 0)
         return EP_ERR_INVALID_ARG;
     cudaStream_t stream = static_cast<cudaStream_t>(stream_);
-    const int T = shape->num_tokens, K = shape->top_k, vpr = shape->hidden / 8;
-    const GroupPlan p = plan_group(vpr);
-    const int grid = ceil_div(T, p.rows_per_block);
-    reduce_to_rows_kernel<<<grid, p.block, 0, stream>>>(static_cast<const uint4 *>(out), out_rows, pair_slot, recv_slot,
-                                                        nullptr, topk_weights, static_cast<uint4 *>(partial),
-                                                        partial_capacity_rows, T, K, shape->num_experts,
-                                                        shape->num_ranks, vpr, p.G, status);
-    sum_rows_kernel<<<grid, p.block, 0, stream>>>(static_cast<const uint4 *>(partial), partial_capacity_rows, recv_slot,
-                                                  static_cast<uint4 *>(y), T, K, vpr, p.G, status);
-    EP_LAUNCH_CHECK(2);
-    return EP_OK;
+    rc = launch_partial_rows(*shape, out, out_rows, pair_slot, recv_slot, topk_weights, partial, partial_capacity_rows,
+                             status, stream);
+    if (rc != EP_OK) return rc;
+    return launch_sum_partial_rows(shape->hidden, shape->top_k, partial, partial_capacity_rows, recv_slot, y,
+                                   shape->num_tokens, status, stream);
 }
 
 extern "C" int ep_dense_allgather(const ep_shape_t *shape, const void *x, void *gathered, void *stream_)
