@@ -541,6 +541,79 @@ def host_staged_arms(ep, wl, iters=10, sweep=True):
     for name, fl in [("flags in device memory", flags_dev), ("flags in pinned host memory", flags_pin)]:
         waits[name] = {"us": timed(lambda: ep.ep_wait_senders(fl, n_s, 3, 100_000_000)) * 1e3, "senders": n_s}
     res["flag_wait_posted"] = waits
+
+    # combine return leg: per-rank partial rows up, down to the owner, summed on the SMs
+    so_host = lay.src_row_offsets.cpu()
+    son = so_host.numpy()
+    local_rows = int(sum(son[r, r + 1] - son[r, r] for r in range(R)))
+    y = torch.empty(cfg.T, cfg.H, dtype=torch.bfloat16, device=dev)
+    D, P, L = ep.HOST_DUPLEX, ep.HOST_PER_PEER, ep.HOST_LOCAL_ON_DEVICE
+    legs = {}
+    for name, fl in [("serial, one reduction behind the last download", 0), ("duplex, one reduction", D),
+                     ("duplex, reduction per owner", D | P),
+                     ("duplex, reduction per owner, local blocks stay on the device", D | P | L)]:
+        best = 1e30
+        for rnd in range(iters + 1):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(up)
+            ep.ep_host_combine(wl.out, lay, wl.w, so_host, staging, back, bounce, y, E, R, round=rnd, flags=fl,
+                               stream_up=up, stream_down=down)
+            b.record(down)
+            torch.cuda.synchronize()
+            best = min(best, a.elapsed_time(b))
+        rows = n_recv - (local_rows if fl & L else 0)
+        legs[name] = {"us": best * 1e3, "rows_over_link": rows, "GB/s_each_way": rows * row / (best * 1e-3) / 1e9,
+                      "frac_of_d2h_probe": rows * row / (best * 1e-3) / 1e9 / d2h,
+                      "frac_of_h2d_probe": rows * row / (best * 1e-3) / 1e9 / h2d, "tokens/s": cfg.T / (best * 1e-3)}
+    res["combine_return_leg"] = legs
+
+    # dispatch with one consumer per sender: when is the first sender's data in use, when the last
+    grouped = torch.empty(cfg.T * cfg.K, cfg.H, dtype=torch.bfloat16, device=dev)
+    stamps = torch.zeros(R + 1, dtype=torch.int64, device=dev)
+    cons = torch.cuda.Stream()
+    t0 = time.perf_counter()
+    so_timed = lay.src_row_offsets.cpu()                 # the segment table's trip to the host, timed once
+    fetch_us = (time.perf_counter() - t0) * 1e6
+    per_sender = {"src_row_offsets_to_host_us": fetch_us}
+    for name, fl in [("consumer per sender", D | P), ("consumers behind the last download", D)]:
+        firsts, lasts = [], []
+        for rnd in range(iters + 1):
+            ep.ep_host_dispatch_per_sender(x, lay, so_timed, staging, back, bounce, grouped, E, R, round=rnd, flags=fl,
+                                           stamps_ns=stamps, stream_up=up, stream_down=down, stream_consume=cons)
+            torch.cuda.synchronize()
+            st = stamps.cpu().numpy()
+            firsts.append((st[1] - st[0]) * 1e-3)
+            lasts.append((st[-1] - st[0]) * 1e-3)
+        per_sender[name] = {"first_sender_consumed_us": float(np.median(firsts[1:])),
+                            "all_senders_consumed_us": float(np.median(lasts[1:]))}
+    res["dispatch_per_sender"] = per_sender
+    del grouped
+
+    # consecutive rounds (dispatch round trip, then combine return leg): with the caller's per-half events
+    # round n+1's uploads overlap round n's downloads; without, every call waits for the download stream
+    bounce2 = torch.empty(2 * cap, cfg.H, dtype=torch.bfloat16).pin_memory()
+    back2 = torch.empty(cap, cfg.H, dtype=torch.bfloat16, device=dev)
+    send2 = torch.empty(cap, cfg.H, dtype=torch.bfloat16, device=dev)
+    n_rounds = 6
+    rounds = {}
+    for name, overlap in [("rounds ordered by the download stream", False), ("rounds overlapped (per-half events)", True)]:
+        best = 1e30
+        for _ in range(3):
+            hf1, hf2 = (ep.HalfFreeEvents(), ep.HalfFreeEvents()) if overlap else (None, None)
+            torch.cuda.synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(up)
+            for rnd in range(n_rounds):
+                ep.ep_host_roundtrip(x, lay.recv_slot, offs_host, staging, bounce, back, E, R, round=rnd, chunks_per_rank=1,
+                                     duplex=True, stream_up=up, stream_down=down, half_free=hf1)
+                ep.ep_host_combine(wl.out, lay, wl.w, so_host, send2, back2, bounce2, y, E, R, round=rnd, flags=D | P,
+                                   stream_up=up, stream_down=down, half_free=hf2)
+            b.record(down)
+            torch.cuda.synchronize()
+            best = min(best, a.elapsed_time(b))
+        rounds[name] = {"us_per_round": best * 1e3 / n_rounds, "rounds": n_rounds,
+                        "GB/s_each_way": 2 * n_recv * row * n_rounds / (best * 1e-3) / 1e9}
+    res["dispatch_plus_combine_rounds"] = rounds
     return res
 
 

@@ -26,7 +26,9 @@
  *     [expert_offsets[r*E/R], expert_offsets[(r+1)*E/R])
  *
  * Every function returns EP_OK (0) or a negative ep_error_t. No function
- * allocates device memory, prints, throws or aborts. Unless stated otherwise a
+ * allocates device memory, prints, throws or aborts. State the library keeps
+ * between calls: the last CUDA error code, a launch counter, per-device one-time
+ * kernel attributes, and the event pool of the multi-stream host-staged calls. Unless stated otherwise a
  * function only enqueues work on `stream` (a cudaStream_t passed as void*; NULL
  * is the default stream) and does not synchronise. "device" pointers must be
  * valid on the current CUDA device; the caller owns every buffer.
@@ -244,24 +246,112 @@ int ep_dispatch_copy_engine(const ep_shape_t *shape, const void *x, const int32_
                             void *stream);
 
 /*
- * Host-staged round trip with separate upload and download streams (Section
- * 4.3: uploads and downloads are issued on two different streams and cut into
- * chunks so that both directions of the host link are busy; Section 4.4: two alternating bounce
- * buffers). Packs the receive rows into `staging` (device) with the dispatch
- * kernel on stream_up, copies them chunk by chunk to the bounce buffer
- * (pinned host, 2 * staging_capacity_rows rows: half `round & 1` is used) and
- * from there into `recv` (device, same row layout) on stream_down. Each rank's
- * partition is cut into chunks_per_rank chunks. duplex != 0: a chunk's download
- * is released by an event right after its upload, so uploads and downloads
- * overlap; duplex == 0: all uploads, then all downloads. The result is complete
- * when stream_down is; stream_up first waits for what is queued on stream_down.
- * rank_row_offsets_host (host, [R+1]) must hold the layout's offsets. Events are
- * created on first use and kept (no device memory is allocated).
+ * Host-staged transfers on two streams: shared conventions of ep_host_roundtrip,
+ * ep_host_dispatch_per_sender and ep_host_combine.
+ *
+ *   - Bounce buffer (Section 4.2: the pinned host buffer every device writes once
+ *     and the others read; Section 4.4: two buffers alternate): bounce_host is
+ *     pinned host memory of 2 * capacity_rows rows of H bf16; a call uses the half
+ *     `round & 1`, at the same row offsets as the device buffers.
+ *   - Streams (Section 4.3: uploads and downloads are issued on two different
+ *     streams and cut into pieces, so that both directions of the host link are
+ *     busy): device-to-host copies and the packing / partial-sum kernel run on
+ *     stream_up, host-to-device copies and what consumes them on stream_down (and
+ *     stream_consume). Inputs must be complete on stream_up; results are complete
+ *     when stream_down (and stream_consume) are.
+ *   - Reuse of a half (Section 4.4: a buffer is reused only after its readers are
+ *     done with it): half_free_events is NULL or an array of two cudaEvent_t the
+ *     caller created (passed as void*). Given, a call waits on stream_up for
+ *     half_free_events[round & 1] before it writes the half and records that event
+ *     on stream_down after its last read of it; so round n+1's uploads overlap
+ *     round n's downloads and round n+2 waits for round n. An event that was never
+ *     recorded counts as complete. NULL: the call's uploads wait for everything
+ *     queued on stream_down (no overlap between rounds, always safe).
+ *   - flags: EP_HOST_DUPLEX            a piece's download is released by an event right after
+ *                                      its upload (else: all uploads, then all downloads);
+ *            EP_HOST_PER_PEER          the consumer is launched per peer rank as soon as that
+ *                                      peer's pieces are down (Section 4.4, per-sender policy),
+ *                                      else once behind the last download (global policy);
+ *            EP_HOST_LOCAL_ON_DEVICE   a segment whose two ranks coincide is copied on the
+ *                                      device and never crosses the host link (Section 4.2:
+ *                                      only the N-1 remote shards / blocks travel).
+ *   - Process-wide state: the ordering events between the streams come from a pool
+ *     the library creates on first use, per device, and keeps until the process
+ *     exits (events hold no device memory). A call holds the pool's lock while it
+ *     enqueues, so calls from several host threads are serialised, not interleaved.
+ *     The same holds for ep_host_step_pipelined.
+ */
+#define EP_HOST_DUPLEX          1
+#define EP_HOST_PER_PEER        2
+#define EP_HOST_LOCAL_ON_DEVICE 4
+
+/*
+ * Host-staged dispatch round trip. Packs the receive rows into `staging` (device)
+ * with the dispatch kernel on stream_up, copies them piece by piece to the bounce
+ * half and from there into `recv` (device, same row layout) on stream_down. Each
+ * rank's partition [rank_row_offsets_host[r], [r+1]) (host, [R+1]) is cut into
+ * chunks_per_rank pieces (1..64). duplex != 0: EP_HOST_DUPLEX as above.
+ * Errors: EP_ERR_CAPACITY when the offsets exceed staging_capacity_rows.
  */
 int ep_host_roundtrip(const ep_shape_t *shape, const void *x, const int32_t *recv_slot,
                       const int32_t *rank_row_offsets_host, void *staging, int64_t staging_capacity_rows,
                       void *bounce_host, int round, void *recv, int chunks_per_rank, int duplex,
-                      int32_t *status, void *stream_up, void *stream_down);
+                      int32_t *status, void *stream_up, void *stream_down, void *const *half_free_events);
+
+/*
+ * Host-staged dispatch with per-sender completion (Section 4.4: a receiver starts
+ * on each sender's data as soon as that sender is done; Section 4.5: computation
+ * on a sender's activations begins while the other senders' transfers continue).
+ * The pieces are the (destination r, sender s) segments
+ * [src_row_offsets_host[r][s], [r][s+1]) of the receive space (host copy of the
+ * layout's src_row_offsets, [R][R+1]), moved sender by sender. The consumer of
+ * sender s is the local grouping of the pairs of s's tokens,
+ *   grouped[pair_slot[t][k]] = recv[recv_slot[t][k]]  for t in s's block,
+ * on stream_consume. EP_HOST_PER_PEER: it is launched behind sender s's last
+ * download; otherwise all R consumers are launched behind the last download of
+ * all. After the call recv holds the dispatched rows and grouped equals what
+ * ep_group produces.
+ *   sender_flags  NULL, or R completion flags (device or mapped pinned memory):
+ *                 the consumer of sender s is additionally gated by a bounded wait
+ *                 (as ep_wait_senders: epoch, timeout_ns <= 2 s, EP_STATUS_TIMEOUT
+ *                 and fall through when it runs out) on sender_flags[s]; arrived
+ *                 (device, [R], may be NULL) receives the epoch per sender. The
+ *                 flags are written by the host or by earlier work; the library
+ *                 never makes a kernel wait on a kernel it launches later.
+ *   stamps_ns     NULL, or R+1 device words: [0] = global timer (ns) when the
+ *                 pipeline starts on stream_up, [1+s] = when sender s's consumer
+ *                 has finished.
+ */
+int ep_host_dispatch_per_sender(const ep_shape_t *shape, const void *x, const int32_t *recv_slot,
+                                const int32_t *pair_slot, const int32_t *src_row_offsets_host, void *staging,
+                                void *recv, int64_t capacity_rows, void *bounce_host, int round, void *grouped,
+                                int64_t grouped_capacity_rows, const uint32_t *sender_flags, uint32_t epoch,
+                                uint64_t timeout_ns, uint32_t *arrived, uint64_t *stamps_ns, int flags,
+                                int32_t *status, void *stream_up, void *stream_down, void *stream_consume,
+                                void *const *half_free_events);
+
+/*
+ * Host-staged combine, the return leg (Section 4.2, reduce-scatter with GPU
+ * reduction: every device uploads the blocks meant for the others, every owner
+ * downloads the blocks meant for it and adds them on its SMs; Section 4.3: the
+ * reduction stays on an SM; Section 4.4, Figure 10: an owner starts as soon as its
+ * senders are done). Computes exactly what ep_combine_partial computes:
+ *   1. on stream_up, every expert rank sums its weighted outputs per token it
+ *      received into one row of partial_send (receive space, device);
+ *   2. the (expert rank r, owner s) blocks [src_row_offsets_host[r][s], [r][s+1])
+ *      travel owner by owner: device -> bounce half on stream_up, bounce half ->
+ *      partial_recv (device) on stream_down;
+ *   3. on stream_down the owner adds a token's partial rows into y:
+ *      EP_HOST_PER_PEER: per owner s as soon as its R blocks are down; otherwise
+ *      once for all tokens behind the last download.
+ * partial_send, partial_recv: [partial_capacity_rows][H] bf16 device buffers;
+ * afterwards partial_recv equals the `partial` of ep_combine_partial and y its y.
+ */
+int ep_host_combine(const ep_shape_t *shape, const void *out, int64_t out_rows, const int32_t *pair_slot,
+                    const int32_t *recv_slot, const float *topk_weights, const int32_t *src_row_offsets_host,
+                    void *partial_send, void *partial_recv, int64_t partial_capacity_rows, void *bounce_host,
+                    int round, void *y, int flags, int32_t *status, void *stream_up, void *stream_down,
+                    void *const *half_free_events);
 
 /*
  * Per-sender completion flags (Section 4.4: the payload stays contiguous and the
@@ -303,7 +393,9 @@ int ep_host_step(const ep_shape_t *shape, const void *x_host, const int32_t *top
  * whole routing table, before the first chunk). Results are identical to
  * ep_host_step. Complete when stream_out is. The three streams must differ for
  * any overlap; the arena may be reused by the next call without synchronising
- * (the call orders itself after the previous one). 1 <= chunks <= 256.
+ * (the call orders itself after the previous one). 1 <= chunks <= 256. Ordering
+ * events come from the library's process-wide pool (see the host-staged
+ * conventions above); calls from several host threads are serialised.
  */
 int ep_host_step_pipelined(const ep_shape_t *shape, const void *x_host, const int32_t *topk_idx_host,
                            const float *topk_weights_host, void *y_host, int32_t *status_host, void *arena,

@@ -25,7 +25,7 @@ void count_launches(int n);                // feeds ep_launch_count
 // Ordering events of the multi-stream entry points: *pool gets at least `need` timing-free events of
 // the current device; `hold` owns the pool's mutex until the caller lets go of it (after its last
 // record/wait has been enqueued). At most kOrderEventPool events per call.
-constexpr int kOrderEventPool = 1024;
+constexpr int kOrderEventPool = 4352;   // 64*64 segments plus per-rank and per-call events
 int order_events(cudaEvent_t **pool, int need, std::unique_lock<std::mutex> &hold);
 
 #define EP_CUDA_TRY(expr)                                   \

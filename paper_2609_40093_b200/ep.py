@@ -20,11 +20,12 @@ STATUS_BAD_INDEX = 1
 STATUS_CAPACITY = 2
 STATUS_TIMEOUT = 4
 PROBE_READ, PROBE_WRITE, PROBE_COPY, PROBE_MEMCPY = 0, 1, 2, 3
+HOST_DUPLEX, HOST_PER_PEER, HOST_LOCAL_ON_DEVICE = 1, 2, 4
 
 EXPORTS = [
     "ep_layout_workspace_bytes", "ep_layout", "ep_layout_ranks", "ep_layout_pairs", "ep_layout_static", "ep_layout_static_scratch_bytes", "ep_dispatch", "ep_combine", "ep_group",
     "ep_combine_partial", "ep_dense_allgather", "ep_dense_reduce_scatter",
-    "ep_host_roundtrip", "ep_wait_senders", "ep_post_flags", "ep_host_step_pipelined",
+    "ep_host_roundtrip", "ep_host_dispatch_per_sender", "ep_host_combine", "ep_wait_senders", "ep_post_flags", "ep_host_step_pipelined",
     "ep_dispatch_copy_engine", "ep_host_step_arena_bytes", "ep_host_step", "ep_status",
     "ep_probe_bandwidth", "ep_launch_count", "ep_strerror", "ep_last_cuda_error",
 ]
@@ -76,7 +77,10 @@ def lib() -> ctypes.CDLL:
         L.ep_combine_partial.argtypes = [sp, vp, i64, vp, vp, vp, vp, i64, vp, vp, vp]
         L.ep_dense_allgather.argtypes = [sp, vp, vp, vp]
         L.ep_dense_reduce_scatter.argtypes = [sp, vp, vp, i64, vp, vp, vp, vp, vp, vp]
-        L.ep_host_roundtrip.argtypes = [sp, vp, vp, vp, vp, i64, vp, i32, vp, i32, i32, vp, vp, vp]
+        L.ep_host_roundtrip.argtypes = [sp, vp, vp, vp, vp, i64, vp, i32, vp, i32, i32, vp, vp, vp, vp]
+        L.ep_host_dispatch_per_sender.argtypes = [sp, vp, vp, vp, vp, vp, vp, i64, vp, i32, vp, i64, vp, ctypes.c_uint32,
+                                                  ctypes.c_uint64, vp, vp, i32, vp, vp, vp, vp, vp]
+        L.ep_host_combine.argtypes = [sp, vp, i64, vp, vp, vp, vp, vp, vp, i64, vp, i32, vp, i32, vp, vp, vp, vp]
         L.ep_wait_senders.argtypes = [vp, i32, ctypes.c_uint32, ctypes.c_uint64, vp, vp, vp]
         L.ep_post_flags.argtypes = [vp, i32, i32, ctypes.c_uint32, vp]
         L.ep_dispatch_copy_engine.argtypes = [sp, vp, vp, vp, vp, i64, vp, vp, vp]
@@ -92,7 +96,7 @@ def lib() -> ctypes.CDLL:
         L.ep_strerror.argtypes = [i32]
         for name in ["ep_layout", "ep_dispatch", "ep_combine", "ep_group", "ep_dispatch_copy_engine",
                      "ep_combine_partial", "ep_dense_allgather", "ep_dense_reduce_scatter",
-                     "ep_host_roundtrip", "ep_wait_senders", "ep_post_flags",
+                     "ep_host_roundtrip", "ep_host_dispatch_per_sender", "ep_host_combine", "ep_wait_senders", "ep_post_flags",
                      "ep_host_step", "ep_status", "ep_probe_bandwidth", "ep_last_cuda_error"]:
             getattr(L, name).restype = i32
         _lib = L
@@ -275,19 +279,70 @@ def ep_dispatch_copy_engine(x, recv_slot, staging, recv_host, E, R, rank_row_off
     return recv_host
 
 
+def _sp(stream):
+    return ctypes.c_void_p(stream.cuda_stream) if stream is not None else _stream()
+
+
+class HalfFreeEvents:
+    """Two caller-owned CUDA events, one per half of a two-half bounce buffer, in the form the
+    host-staged calls take them (an array of two cudaEvent_t). torch creates an event's handle
+    when it is first recorded, so both are recorded once on the current stream here."""
+
+    def __init__(self):
+        self.events = [torch.cuda.Event(), torch.cuda.Event()]
+        for e in self.events:
+            e.record()
+        self.array = (ctypes.c_void_p * 2)(*[ctypes.c_void_p(e.cuda_event) for e in self.events])
+
+
+def _half_free(h):
+    return None if h is None else ctypes.cast(h.array, ctypes.c_void_p)
+
+
 def ep_host_roundtrip(x, recv_slot, rank_row_offsets_host, staging, bounce_host, recv, E, R, round=0,
-                      chunks_per_rank=1, duplex=True, status=None, stream_up=None, stream_down=None):
+                      chunks_per_rank=1, duplex=True, status=None, stream_up=None, stream_down=None,
+                      half_free: HalfFreeEvents = None):
     """Pack -> upload to the pinned bounce buffer -> download into `recv`, on two streams
     (torch.cuda.Stream objects; default: the current stream for both)."""
     T, H = x.shape
     K = recv_slot.shape[1]
-    up = ctypes.c_void_p(stream_up.cuda_stream) if stream_up is not None else _stream()
-    down = ctypes.c_void_p(stream_down.cuda_stream) if stream_down is not None else _stream()
     _check(lib().ep_host_roundtrip(ctypes.byref(_shape(T, K, H, E, R)), _ptr(x), _ptr(recv_slot),
                                    _ptr(rank_row_offsets_host), _ptr(staging), staging.shape[0], _ptr(bounce_host),
-                                   int(round), _ptr(recv), int(chunks_per_rank), int(bool(duplex)), _ptr(status), up, down),
+                                   int(round), _ptr(recv), int(chunks_per_rank), int(bool(duplex)), _ptr(status),
+                                   _sp(stream_up), _sp(stream_down), _half_free(half_free)),
            "ep_host_roundtrip")
     return recv
+
+
+def ep_host_dispatch_per_sender(x, lay: Layout, src_row_offsets_host, staging, recv, bounce_host, grouped, E, R,
+                                round=0, flags=HOST_DUPLEX | HOST_PER_PEER, sender_flags=None, epoch=0,
+                                timeout_ns=0, arrived=None, stamps_ns=None, status=None, stream_up=None,
+                                stream_down=None, stream_consume=None, half_free: HalfFreeEvents = None):
+    """Host-staged dispatch moved sender by sender, the local grouping of each sender's pairs
+    launched as that sender's rows arrive. src_row_offsets_host: CPU int32 [R, R+1]."""
+    T, H = x.shape
+    K = lay.recv_slot.shape[1]
+    _check(lib().ep_host_dispatch_per_sender(
+        ctypes.byref(_shape(T, K, H, E, R)), _ptr(x), _ptr(lay.recv_slot), _ptr(lay.pair_slot),
+        _ptr(src_row_offsets_host), _ptr(staging), _ptr(recv), staging.shape[0], _ptr(bounce_host), int(round),
+        _ptr(grouped), grouped.shape[0], _ptr(sender_flags), int(epoch), int(timeout_ns), _ptr(arrived),
+        _ptr(stamps_ns), int(flags), _ptr(status), _sp(stream_up), _sp(stream_down), _sp(stream_consume),
+        _half_free(half_free)), "ep_host_dispatch_per_sender")
+    return grouped
+
+
+def ep_host_combine(out, lay: Layout, topk_weights, src_row_offsets_host, partial_send, partial_recv, bounce_host, y,
+                    E, R, round=0, flags=HOST_DUPLEX | HOST_PER_PEER, status=None, stream_up=None, stream_down=None,
+                    half_free: HalfFreeEvents = None):
+    """Host-staged combine: per-rank partial rows up to the bounce buffer, down to the owner, summed on the SMs."""
+    T, K = lay.pair_slot.shape
+    H = out.shape[1]
+    _check(lib().ep_host_combine(
+        ctypes.byref(_shape(T, K, H, E, R)), _ptr(out), out.shape[0], _ptr(lay.pair_slot), _ptr(lay.recv_slot),
+        _ptr(topk_weights), _ptr(src_row_offsets_host), _ptr(partial_send), _ptr(partial_recv), partial_send.shape[0],
+        _ptr(bounce_host), int(round), _ptr(y), int(flags), _ptr(status), _sp(stream_up), _sp(stream_down),
+        _half_free(half_free)), "ep_host_combine")
+    return y
 
 
 def ep_wait_senders(flags, num_senders: int, epoch: int, timeout_ns: int, arrived=None, status=None):
