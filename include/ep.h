@@ -343,7 +343,8 @@ int ep_host_dispatch_per_sender(const ep_shape_t *shape, const void *x, const in
  *      partial_recv (device) on stream_down;
  *   3. on stream_down the owner adds a token's partial rows into y:
  *      EP_HOST_PER_PEER: per owner s as soon as its R blocks are down; otherwise
- *      once for all tokens behind the last download.
+ *      once for all tokens behind the last download (then, unless local blocks
+ *      stay on the device, an expert rank's R blocks travel as one piece).
  * partial_send, partial_recv: [partial_capacity_rows][H] bf16 device buffers;
  * afterwards partial_recv equals the `partial` of ep_combine_partial and y its y.
  */

@@ -2,11 +2,12 @@
 //
 // The work is a stable counting sort of the T*K (token, k) pairs by expert id plus
 // a stable count of the distinct (token, rank) hits. Determinism never depends on
-// the arrival order of atomics: tokens are cut into contiguous tiles of 32*m
-// tokens, one warp owns a tile, a CTA owns `warps` consecutive tiles, and every
-// rank inside a tile comes from warp ballots / matches whose lane order is the
-// (t,k) order. Every CTA
-//   1. histograms its tiles (experts, rank hits, bad ids) in shared memory,
+// the arrival order of atomics between warps: tokens are cut into contiguous tiles
+// of 32*m tokens, one warp owns a tile, a CTA owns `warps` consecutive tiles, and
+// every rank inside a tile comes from warp ballots / matches whose lane order is
+// the (t,k) order. Every CTA
+//   1. histograms its tiles (experts, rank hits, bad ids) in shared memory, one
+//      private histogram per warp,
 //   2. learns, per bin, the count in earlier CTAs and the grand total,
 //   3. scans the totals over bins (expert_offsets, rank_row_offsets),
 //   4. replays its tiles in (t,k) order with running counters that start at
@@ -17,12 +18,22 @@
 //   cluster  up to 8 CTAs of 8 warps (up to 2048 tokens) form one thread-block cluster
 //            and read each other's CTA totals through distributed shared memory
 //            between two cluster barriers: one launch, no global scratch;
-//   global   larger batches, spread over up to 128 CTAs of 8 warps because the replay
-//            is throughput-bound per SM: a first kernel writes cta_part[cta][bin] to
-//            the workspace; the main kernel, launched with programmatic stream
+//   global   larger batches, or a device that cannot keep the cluster resident: up to
+//            128 CTAs of 8 warps, because the replay's scattered 4-byte stores (two per
+//            pair) are bound per SM (at T=8192, K=8: 8 CTAs of 32 warps 24 us, 32 CTAs of
+//            8 warps 15 us); a first kernel writes cta_part[cta][bin] to the
+//            workspace; the main kernel, launched with programmatic stream
 //            serialisation so that its histogram phase overlaps the first kernel,
 //            executes griddepcontrol.wait and then reads every cta_part row.
 // Bins: [0,E) experts, [E,E+R) rank hits, [E+R] ids outside [-1,E).
+//
+// Inner loops: the ids of 32 tokens are staged in shared memory with an odd row
+// stride (token-per-lane and pair-per-lane accesses are both free of bank
+// conflicts); divisions by E/R and K are one 32-bit high multiply; a rank's ballot
+// is kept by lane r, so the R ballots of a group cost R votes and no serial
+// section; the running counter of an expert is advanced by one shared-memory
+// atomic of the group's first lane (the counters are private to the warp, so their
+// order is the program order of that warp).
 #include <cooperative_groups.h>
 
 #include <atomic>
@@ -36,7 +47,7 @@ namespace ep {
 namespace {
 
 constexpr int kMaxWarpsSingle = 32;     // one CTA holds every tile: up to 1024 tokens
-constexpr int kMaxWarps = 8;            // tiles per CTA otherwise (the replay is throughput-bound per SM: spread it)
+constexpr int kMaxWarps = 8;            // warps per CTA otherwise (the replay's scattered stores are bound per SM: spread it)
 constexpr int kMaxCluster = 8;          // portable cluster size
 constexpr int kMaxCtasGlobal = 128;
 constexpr size_t kSmemBudget = 200 * 1024;
@@ -55,9 +66,9 @@ struct LayoutPlan {
     size_t workspace_bytes;
 };
 
-// shared memory: per warp  hist[bins] | ballots[kMaxRanks] | slots[32*K] | ids[32*K];
-//                per CTA   tot_e[E+1] | tot_r[R+1] | pre[bins] | cta_tot[bins] | scan[32]
-inline size_t per_warp_ints(int bins, int K) { return (size_t)bins + kMaxRanks + 64 * (size_t)K; }
+// shared memory: per warp  hist[bins] | ballots[kMaxRanks] | rows[32][Kp] | ids[32][Kp]   (Kp = K | 1);
+//                per CTA   tot[bins+1] | pre[bins] | cta_tot[bins] | scan[32]
+inline size_t per_warp_ints(int bins, int K) { return (size_t)bins + kMaxRanks + 64 * (size_t)(K | 1); }
 inline size_t per_cta_ints(int bins) { return 3 * (size_t)bins + 2 + 32; }
 
 LayoutPlan make_plan(const ep_shape_t &s)
@@ -107,76 +118,111 @@ __device__ __forceinline__ int fdiv(int n, const FastDiv &f)
 {
     return f.d == 1 ? n : (int)__umul64hi((uint64_t)(uint32_t)n, f.m);
 }
-
+// n / d by one 32-bit high multiply with mul = ceil(2^32 / d) (0 stands for d == 1): exact while
+// n * d < 2^32, which holds for an expert id over E/R (both <= 4096) and a pair index of a group over K.
+inline uint32_t small_div_mul(int d) { return d > 1 ? 0xffffffffu / (uint32_t)d + 1u : 0u; }
+__device__ __forceinline__ int sdiv(int n, uint32_t mul) { return mul ? (int)__umulhi((uint32_t)n, mul) : n; }
 
 struct LayoutArgs {
     const int32_t *idx;
     ep_layout_t out;
     int32_t *cta_part;  // [n_ctas][bins], global form only
-    int T, K, E, R, Tr;
-    FastDiv by_El, by_K, by_Tr;
+    int T, K, Kp, E, R, Tr;
+    uint32_t mul_El, mul_K;
+    FastDiv by_Tr;
     int tile_tokens, n_tiles, bins, n_ctas, mode;
     int parts;   // kPartRanks | kPartPairs: which outputs this call writes
     int blo;     // first bin in use: 0, or E when only the receive-row half is wanted
 };
 
-// The warp copies the expert ids of the 32 tokens [tb, tb+32) into ids[32*K] (coalesced, all loads in
-// flight at once); entries of tokens >= t1 become -1. Returns the number of live items.
+// The warp copies the expert ids of the 32 tokens [tb, tb+32) into ids[32][Kp] (coalesced, eight loads
+// per lane in flight before the first use); entries of tokens >= t1 become -1. Returns the number of live items.
 __device__ __forceinline__ int stage_group(const LayoutArgs &a, int32_t *ids, int tb, int t1, int lane)
 {
     const int n_items = (min(t1, tb + 32) - tb) * a.K;
     const int32_t *src = a.idx + (size_t)tb * a.K;
-    for (int i = lane; i < 32 * a.K; i += 32) ids[i] = i < n_items ? __ldg(src + i) : -1;
+    for (int base = lane; base < 32 * a.K; base += 256) {
+        int32_t v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int i = base + 32 * u;
+            v[u] = i < n_items ? __ldg(src + i) : -1;
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int i = base + 32 * u;
+            if (i < 32 * a.K) {
+                const int tok = sdiv(i, a.mul_K);
+                ids[tok * a.Kp + (i - tok * a.K)] = v[u];
+            }
+        }
+    }
     __syncwarp();
     return n_items;
 }
 
-// rank bitmask of the token this lane owns in the staged group
-__device__ __forceinline__ unsigned long long token_rank_mask(const LayoutArgs &a, const int32_t *ids, int lane)
+// position in ids[] / rows[] of pair i (in (t,k) order) of the staged group
+__device__ __forceinline__ int pair_pos(const LayoutArgs &a, int i)
+{
+    const int tok = sdiv(i, a.mul_K);
+    return tok * a.Kp + (i - tok * a.K);
+}
+
+// rank bitmask of the token this lane owns in the staged group; *bad counts ids outside [-1, E)
+__device__ __forceinline__ unsigned long long token_rank_mask(const LayoutArgs &a, const int32_t *ids, int lane, int *bad)
 {
     unsigned long long mask = 0ull;
     for (int k = 0; k < a.K; ++k) {
-        const int e = ids[lane * a.K + k];
-        if (e >= 0 && e < a.E) mask |= 1ull << fdiv(e, a.by_El);
+        const int e = ids[lane * a.Kp + k];
+        if (e >= 0 && e < a.E) mask |= 1ull << sdiv(e, a.mul_El);
+        else if (e != -1) ++*bad;
     }
     return mask;
 }
 
 // One warp counts its tile into hist[bins]. kShared == false: hist is this warp's own and is
 // zeroed here; kShared == true: hist is one histogram for the whole CTA, zeroed by the caller.
+// Returns the rank mask of this lane's token in the tile's last group (reused by a one-group replay).
 template <bool kShared>
-__device__ __forceinline__ void count_tile(const LayoutArgs &a, int32_t *hist, int32_t *ids, int tile, int lane)
+__device__ __forceinline__ unsigned long long count_tile(const LayoutArgs &a, int32_t *hist, int32_t *ids, int tile, int lane)
 {
     if (!kShared) {
         for (int b = a.blo + lane; b < a.bins; b += 32) hist[b] = 0;
         __syncwarp();
     }
-    if (tile >= a.n_tiles) return;
+    if (tile >= a.n_tiles) return 0ull;
     const int t0 = tile * a.tile_tokens;
     const int t1 = min(a.T, t0 + a.tile_tokens);
     int bad = 0;
+    int hits0 = 0, hits1 = 0;                        // lane l counts the hits of ranks l and l + 32
+    unsigned long long mask = 0ull;
     for (int tb = t0; tb < t1; tb += 32) {
-        const int n_items = stage_group(a, ids, tb, t1, lane);
-        for (int i = lane; i < n_items; i += 32) {                   // experts: any order
-            const int e = ids[i];
-            if (e >= 0 && e < a.E) {
-                if (a.blo == 0) atomicAdd(hist + e, 1);
-            } else if (e != -1) {
-                ++bad;
+        stage_group(a, ids, tb, t1, lane);
+        if (a.blo == 0)                               // experts: any order
+            for (int k = 0; k < a.K; ++k) {
+                const int e = ids[lane * a.Kp + k];
+                if (e >= 0 && e < a.E) atomicAdd(hist + e, 1);
             }
-        }
-        const unsigned long long mask = token_rank_mask(a, ids, lane);   // rank hits: token per lane, ballot per rank
+        mask = token_rank_mask(a, ids, lane, &bad);   // rank hits: token per lane, ballot per rank
         for (int r = 0; r < a.R; ++r) {
-            const unsigned b = __ballot_sync(kFullMask, (mask >> r) & 1ull);
-            if (lane == 0 && b) {
-                if (kShared) atomicAdd(hist + a.E + r, __popc(b));
-                else hist[a.E + r] += __popc(b);
+            const int c = __popc(__ballot_sync(kFullMask, (mask >> r) & 1ull));
+            if (lane == (r & 31)) {
+                if (r < 32) hits0 += c;
+                else hits1 += c;
             }
         }
         __syncwarp();
     }
+    if (kShared) {
+        if (lane < a.R && hits0) atomicAdd(hist + a.E + lane, hits0);
+        if (lane + 32 < a.R && hits1) atomicAdd(hist + a.E + 32 + lane, hits1);
+    } else {
+        if (lane < a.R) hist[a.E + lane] = hits0;
+        if (lane + 32 < a.R) hist[a.E + 32 + lane] = hits1;
+    }
     if (bad) atomicAdd(hist + a.E + a.R, bad);
     __syncwarp();
+    return mask;
 }
 
 // exclusive scan of v[0..n) in place (shared memory), v[n] = total; whole CTA; sh holds one int per warp
@@ -223,7 +269,7 @@ __global__ void __launch_bounds__(kMaxWarps * 32) layout_cta_count_kernel(Layout
     // one histogram for the CTA (first `bins` words), per-warp id staging behind it
     for (int b = a.blo + threadIdx.x; b < a.bins; b += blockDim.x) smem[b] = 0;
     __syncthreads();
-    count_tile<true>(a, smem, smem + a.bins + warp * 32 * a.K, blockIdx.x * warps + warp, lane);
+    count_tile<true>(a, smem, smem + a.bins + warp * 32 * a.Kp, blockIdx.x * warps + warp, lane);
     __syncthreads();
     int32_t *dst = a.cta_part + (size_t)blockIdx.x * a.bins;
     for (int b = a.blo + threadIdx.x; b < a.bins; b += blockDim.x) dst[b] = smem[b];
@@ -234,12 +280,12 @@ __global__ void __launch_bounds__(kMaxWarpsSingle * 32) layout_assign_kernel(Lay
 {
     extern __shared__ int32_t smem[];
     const int warps = blockDim.x >> 5, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int pw = a.bins + kMaxRanks + 64 * a.K;
+    const int pw = a.bins + kMaxRanks + 64 * a.Kp;
     const int nb = a.E + a.R;
     int32_t *run = smem + warp * pw;                                 // [bins] histogram, later next free slot
     unsigned *bal = reinterpret_cast<unsigned *>(run + a.bins);      // [R] ballots of the current 32 tokens
-    int32_t *slot_s = run + a.bins + kMaxRanks;                      // [32*K] receive slots of the current 32 tokens
-    int32_t *ids = slot_s + 32 * a.K;                                // [32*K] expert ids of the current 32 tokens
+    int32_t *rows = run + a.bins + kMaxRanks;                        // [32][Kp] receive rows of the current 32 tokens
+    int32_t *ids = rows + 32 * a.Kp;                                 // [32][Kp] expert ids of the current 32 tokens
     int32_t *tot = smem + warps * pw;                                // [E+R+1] totals -> one scan: experts, then ranks
     int32_t *pre = tot + a.bins + 1;                                 // [bins] count in earlier CTAs
     int32_t *cta_tot = pre + a.bins;                                 // [bins] this CTA's totals (peers read it)
@@ -247,11 +293,12 @@ __global__ void __launch_bounds__(kMaxWarpsSingle * 32) layout_assign_kernel(Lay
     const int tile = blockIdx.x * warps + warp;
     const unsigned lt = lanemask_lt();
 
-    count_tile<false>(a, run, ids, tile, lane);
+    const unsigned long long mask_kept = count_tile<false>(a, run, ids, tile, lane);
     __syncthreads();
     const bool ranks = a.parts & kPartRanks, pairs = a.parts & kPartPairs;
     for (int b = a.blo + threadIdx.x; b < a.bins; b += blockDim.x) {  // this CTA's total per bin
         int32_t mine = 0;
+#pragma unroll 8
         for (int w = 0; w < warps; ++w) mine += smem[w * pw + b];
         cta_tot[b] = mine;
     }
@@ -304,10 +351,16 @@ __global__ void __launch_bounds__(kMaxWarpsSingle * 32) layout_assign_kernel(Lay
     // next free slot of every bin for every warp: offset + earlier CTAs + earlier warps of this CTA
     for (int b = a.blo + threadIdx.x; b < nb; b += blockDim.x) {
         int32_t running = pre[b] + (b < a.E ? tot[b] : tot[b] - n_pairs);
-        for (int w = 0; w < warps; ++w) {
-            const int32_t v = smem[w * pw + b];
-            smem[w * pw + b] = running;
-            running += v;
+        for (int w0 = 0; w0 < warps; w0 += 8) {                      // eight counts read before the first is replaced
+            int32_t v[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) v[u] = w0 + u < warps ? smem[(w0 + u) * pw + b] : 0;
+#pragma unroll
+            for (int u = 0; u < 8; ++u)
+                if (w0 + u < warps) {
+                    smem[(w0 + u) * pw + b] = running;
+                    running += v[u];
+                }
         }
     }
     __syncthreads();
@@ -319,13 +372,20 @@ __global__ void __launch_bounds__(kMaxWarpsSingle * 32) layout_assign_kernel(Lay
     for (int tb = t0; tb < t1; tb += 32) {
         const int t = tb + lane;
         const bool live = t < t1;
-        // a tile of one 32-token group still has its ids staged from the counting phase
-        const int n_items = a.tile_tokens == 32 ? (min(t1, tb + 32) - tb) * a.K : stage_group(a, ids, tb, t1, lane);
-        // --- receive rows: which of these 32 tokens hit which rank
-        const unsigned long long mask = token_rank_mask(a, ids, lane);
+        // a tile of one 32-token group still has its ids staged (and its rank masks) from the counting phase
+        int n_items, bad = 0;
+        unsigned long long mask;
+        if (a.tile_tokens == 32) {
+            n_items = (min(t1, tb + 32) - tb) * a.K;
+            mask = mask_kept;
+        } else {
+            n_items = stage_group(a, ids, tb, t1, lane);
+            mask = token_rank_mask(a, ids, lane, &bad);
+        }
+        // --- receive rows: which of these 32 tokens hit which rank (lane r keeps rank r's ballot)
         for (int r = 0; r < a.R; ++r) {
             const unsigned b = __ballot_sync(kFullMask, (mask >> r) & 1ull);
-            if (lane == 0) bal[r] = b;
+            if (lane == (r & 31)) bal[r] = b;
         }
         __syncwarp();
         if (live) {
@@ -335,17 +395,17 @@ __global__ void __launch_bounds__(kMaxWarpsSingle * 32) layout_assign_kernel(Lay
                     a.out.src_row_offsets[r * (a.R + 1) + s] = run[a.E + r] + __popc(bal[r] & lt);
             unsigned long long seen = 0ull;
             for (int k = 0; k < a.K; ++k) {
-                const int e = ids[lane * a.K + k];
+                const int e = ids[lane * a.Kp + k];
                 int32_t row = -1;
                 if (e >= 0 && e < a.E) {
-                    const int r = fdiv(e, a.by_El);
+                    const int r = sdiv(e, a.mul_El);
                     row = run[a.E + r] + __popc(bal[r] & lt);
                     if (ranks && !((seen >> r) & 1ull)) {
                         a.out.recv_token[row] = t;
                         seen |= 1ull << r;
                     }
                 }
-                slot_s[lane * a.K + k] = row;
+                rows[lane * a.Kp + k] = row;
             }
         }
         __syncwarp();
@@ -353,7 +413,7 @@ __global__ void __launch_bounds__(kMaxWarpsSingle * 32) layout_assign_kernel(Lay
         __syncwarp();
         int32_t *recv_slot = a.out.recv_slot + (size_t)tb * a.K;
         if (!pairs) {                                // receive-row half only: publish the rows and go on
-            for (int i = lane; i < n_items; i += 32) recv_slot[i] = slot_s[i];
+            for (int i = lane; i < n_items; i += 32) recv_slot[i] = rows[pair_pos(a, i)];
             __syncwarp();
             continue;
         }
@@ -362,25 +422,27 @@ __global__ void __launch_bounds__(kMaxWarpsSingle * 32) layout_assign_kernel(Lay
         for (int j = 0; j < n_items; j += 32) {
             const int i = j + lane;
             const bool act = i < n_items;
-            const int e = act ? ids[i] : -1;
+            const int tok = sdiv(i, a.mul_K);
+            const int pos = tok * a.Kp + (i - tok * a.K);
+            const int e = act ? ids[pos] : -1;
             const bool valid = act && e >= 0 && e < a.E;
             const unsigned m = __match_any_sync(kFullMask, valid ? e : a.E + lane);
+            const int leader = __ffs(m) - 1;
             int32_t first = 0;
+            if (valid && lane == leader) first = atomicAdd(run + e, __popc(m));   // the group's slots, taken at once
+            first = __shfl_sync(kFullMask, first, leader);
             if (valid) {
-                first = run[e];
                 const int32_t p = first + __popc(m & lt);
-                const int32_t row = slot_s[i];
+                const int32_t row = rows[pos];
                 pair_slot[i] = p;
                 if (ranks) recv_slot[i] = row;
-                a.out.pair_token[p] = tb + fdiv(i, a.by_K);
+                a.out.pair_token[p] = tb + tok;
                 a.out.pair_row[p] = row;
             } else if (act) {
                 pair_slot[i] = -1;
                 if (ranks) recv_slot[i] = -1;
             }
-            __syncwarp();
-            if (valid && (m >> lane) <= 1u) run[e] = first + __popc(m);   // highest lane of the group
-            __syncwarp();
+            __syncwarp();                            // orders this step's counter update before the next step's
         }
     }
 }
@@ -458,8 +520,8 @@ int run_layout(const ep_shape_t *shape, const int32_t *topk_idx, const ep_layout
     a.idx = topk_idx;
     a.out = *out;
     a.cta_part = static_cast<int32_t *>(workspace);
-    a.T = T; a.K = shape->top_k; a.E = E; a.R = R; a.Tr = T / R;
-    a.by_El = make_fastdiv(E / R); a.by_K = make_fastdiv(shape->top_k); a.by_Tr = make_fastdiv(T / R);
+    a.T = T; a.K = shape->top_k; a.Kp = shape->top_k | 1; a.E = E; a.R = R; a.Tr = T / R;
+    a.mul_El = small_div_mul(E / R); a.mul_K = small_div_mul(shape->top_k); a.by_Tr = make_fastdiv(T / R);
     a.tile_tokens = plan.tile_tokens; a.n_tiles = plan.n_tiles; a.bins = plan.bins; a.n_ctas = plan.n_ctas;
     a.mode = plan.mode;
     a.parts = parts;

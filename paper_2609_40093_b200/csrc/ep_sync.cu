@@ -211,10 +211,16 @@ struct Trip {
     // phase 0: uploads (and, duplex, the downloads right behind them); phase 1: downloads of the serial form
     int move(int r, int s, int phase)
     {
-        const int64_t a = so[r * (R + 1) + s], b = so[r * (R + 1) + s + 1];
+        return move_rows(so[r * (R + 1) + s], so[r * (R + 1) + s + 1], local_on_device && r == s, phase);
+    }
+    // the same for the whole partition of holder rank r (its R segments are contiguous)
+    int move_partition(int r, int phase) { return move_rows(so[r * (R + 1)], so[r * (R + 1) + R], false, phase); }
+
+    int move_rows(int64_t a, int64_t b, bool local, int phase)
+    {
         if (b <= a) return EP_OK;
         const size_t off = (size_t)a * row_bytes, len = (size_t)(b - a) * row_bytes;
-        if (local_on_device && r == s) {               // holder and peer are the same rank: never crosses the link
+        if (local) {                                   // holder and peer are the same rank: never crosses the link
             if (phase == 0) EP_CUDA_TRY(cudaMemcpyAsync(dst + off, src + off, len, cudaMemcpyDeviceToDevice, up));
             return EP_OK;
         }
@@ -392,6 +398,17 @@ extern "C" int ep_host_combine(const ep_shape_t *shape, const void *out, int64_t
         if (per_owner) return reduce(s, s + 1);
         return s == R - 1 ? reduce(0, R) : EP_OK;
     };
+    if (!per_owner && !trip.local_on_device) {
+        // one reduction at the end and every block over the link: an expert rank's R blocks are contiguous, so
+        // they travel as one piece (R pieces instead of R*R: the fewest that keep both directions busy)
+        for (int phase = 0; phase < (duplex ? 1 : 2); ++phase) {
+            if (phase == 1 && (rc = trip.join()) != EP_OK) return rc;
+            for (int r = 0; r < R; ++r)
+                if ((rc = trip.move_partition(r, phase)) != EP_OK) return rc;
+        }
+        if ((rc = reduce(0, R)) != EP_OK) return rc;
+        return end_round(half_free_events, round, down);
+    }
     for (int s = 0; s < R; ++s) {                // owner-major: every expert rank's block for owner s, then the next owner
         for (int r = 0; r < R; ++r)
             if ((rc = trip.move(r, s, 0)) != EP_OK) return rc;
