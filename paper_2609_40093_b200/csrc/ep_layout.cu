@@ -51,6 +51,7 @@ constexpr int kMaxWarps = 8;            // warps per CTA otherwise (the replay's
 constexpr int kMaxCluster = 8;          // portable cluster size
 constexpr int kMaxCtasGlobal = 128;
 constexpr size_t kSmemBudget = 200 * 1024;
+constexpr int kSteps = 4;               // 32-pair steps of the replay whose latencies overlap
 
 enum { kModeSingle = 0, kModeCluster = 1, kModeGlobal = 2 };
 enum { kPartRanks = 1, kPartPairs = 2 };
@@ -225,10 +226,33 @@ __device__ __forceinline__ unsigned long long count_tile(const LayoutArgs &a, in
     return mask;
 }
 
-// exclusive scan of v[0..n) in place (shared memory), v[n] = total; whole CTA; sh holds one int per warp
+// exclusive scan of v[0..n) in place (shared memory), v[n] = total; whole CTA; sh holds one int per warp.
+// Up to 1024 entries one warp does it alone (a chunk per lane, one shuffle scan, no block barrier inside).
 __device__ void block_exclusive_scan_smem(int32_t *v, int n, int32_t *sh)
 {
     const int nt = blockDim.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nw = nt >> 5;
+    if (n <= 1024) {
+        if (warp == 0) {
+            const int chunk = (n + 31) >> 5;
+            const int lo = min(n, lane * chunk), hi = min(n, lo + chunk);
+            int32_t sum = 0;
+            for (int i = lo; i < hi; ++i) sum += v[i];
+            int32_t incl = sum;
+            for (int off = 1; off < 32; off <<= 1) {
+                const int32_t up = __shfl_up_sync(kFullMask, incl, off);
+                if (lane >= off) incl += up;
+            }
+            int32_t run = incl - sum;
+            for (int i = lo; i < hi; ++i) {
+                const int32_t x = v[i];
+                v[i] = run;
+                run += x;
+            }
+            if (lane == 31) v[n] = incl;
+        }
+        __syncthreads();
+        return;
+    }
     const int chunk = (n + nt - 1) / nt;
     const int lo = min(n, tid * chunk), hi = min(n, lo + chunk);
     int32_t sum = 0;
@@ -419,30 +443,45 @@ __global__ void __launch_bounds__(kMaxWarpsSingle * 32) layout_assign_kernel(Lay
         }
         // --- pair slots: the items of these tokens, 32 at a time in (t,k) order
         int32_t *pair_slot = a.out.pair_slot + (size_t)tb * a.K;
-        for (int j = 0; j < n_items; j += 32) {
-            const int i = j + lane;
-            const bool act = i < n_items;
-            const int tok = sdiv(i, a.mul_K);
-            const int pos = tok * a.Kp + (i - tok * a.K);
-            const int e = act ? ids[pos] : -1;
-            const bool valid = act && e >= 0 && e < a.E;
-            const unsigned m = __match_any_sync(kFullMask, valid ? e : a.E + lane);
-            const int leader = __ffs(m) - 1;
-            int32_t first = 0;
-            if (valid && lane == leader) first = atomicAdd(run + e, __popc(m));   // the group's slots, taken at once
-            first = __shfl_sync(kFullMask, first, leader);
-            if (valid) {
-                const int32_t p = first + __popc(m & lt);
-                const int32_t row = rows[pos];
-                pair_slot[i] = p;
-                if (ranks) recv_slot[i] = row;
-                a.out.pair_token[p] = tb + tok;
-                a.out.pair_row[p] = row;
-            } else if (act) {
-                pair_slot[i] = -1;
-                if (ranks) recv_slot[i] = -1;
+        for (int j0 = 0; j0 < n_items; j0 += 32 * kSteps) {          // kSteps steps of 32 pairs: their matches, then their
+            int pos[kSteps], e[kSteps], leader[kSteps];              // counter updates in order, then their stores
+            unsigned m[kSteps];
+            int32_t first[kSteps];
+#pragma unroll
+            for (int u = 0; u < kSteps; ++u) {
+                const int i = j0 + 32 * u + lane;
+                const int tok = sdiv(i, a.mul_K);
+                pos[u] = tok * a.Kp + (i - tok * a.K);
+                e[u] = i < n_items ? ids[pos[u]] : -1;
+                if (e[u] >= a.E) e[u] = -2;                          // out of range: masked like any negative id
             }
-            __syncwarp();                            // orders this step's counter update before the next step's
+#pragma unroll
+            for (int u = 0; u < kSteps; ++u) {
+                m[u] = __match_any_sync(kFullMask, e[u] >= 0 ? e[u] : a.E + lane);
+                leader[u] = __ffs(m[u]) - 1;
+            }
+#pragma unroll
+            for (int u = 0; u < kSteps; ++u) {
+                first[u] = 0;
+                if (e[u] >= 0 && lane == leader[u]) first[u] = atomicAdd(run + e[u], __popc(m[u]));   // the group's slots at once
+                __syncwarp();                        // orders this step's counter update before the next step's
+            }
+#pragma unroll
+            for (int u = 0; u < kSteps; ++u) {
+                const int i = j0 + 32 * u + lane;
+                first[u] = __shfl_sync(kFullMask, first[u], leader[u]);
+                if (e[u] >= 0) {
+                    const int32_t p = first[u] + __popc(m[u] & lt);
+                    const int32_t row = rows[pos[u]];
+                    pair_slot[i] = p;
+                    if (ranks) recv_slot[i] = row;
+                    a.out.pair_token[p] = tb + sdiv(i, a.mul_K);
+                    a.out.pair_row[p] = row;
+                } else if (i < n_items) {
+                    pair_slot[i] = -1;
+                    if (ranks) recv_slot[i] = -1;
+                }
+            }
         }
     }
 }
