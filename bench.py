@@ -260,7 +260,7 @@ def run_reference(args, cfg):
 class Workload:
     """Device buffers and the step of one configuration."""
 
-    def __init__(self, ep, inputs, cfg, rcfg, dev, seed, serial_layout=False):
+    def __init__(self, ep, inputs, cfg, rcfg, dev, seed, serial_layout=False, separate_calls=False):
         self.ep, self.cfg, self.dev = ep, cfg, dev
         T, K, H, E, R = cfg.T, cfg.K, cfg.H, cfg.E, cfg.R
         d = inputs.make_inputs(rcfg, seed)
@@ -283,6 +283,8 @@ class Workload:
         self.split_layout = (not serial_layout) and not is_small(cfg) and not cfg.host_staged
         self.side = torch.cuda.Stream()
         self.fork_ev, self.join_ev = torch.cuda.Event(), torch.cuda.Event()
+        # decode-size batches: layout and dispatch in one launch (ep_layout_dispatch)
+        self.fused = (not separate_calls) and T <= 1024 and not cfg.host_staged
 
     def step(self, ev=None):
         """layout -> dispatch -> combine. Dispatch needs only the receive-row half of the layout, so for big
@@ -293,7 +295,9 @@ class Workload:
         main = torch.cuda.current_stream()
         if ev:
             ev["t0"].record()
-        if not self.split_layout:
+        if self.fused:
+            ep.ep_layout_dispatch(self.idx, self.x, self.recv, E, R, lay, self.ws)    # one launch for both
+        elif not self.split_layout:
             ep.ep_layout(self.idx, E, R, out=lay, workspace=self.ws)
         else:
             self.fork_ev.record(main)                     # the side stream starts after everything queued so far
@@ -307,7 +311,8 @@ class Workload:
             self.join_ev.record(self.side)
         if ev:
             ev["t1"].record()
-        ep.ep_dispatch(self.x, lay.recv_slot, self.recv, E, R, status=lay.status)
+        if not self.fused:
+            ep.ep_dispatch(self.x, lay.recv_slot, self.recv, E, R, status=lay.status)
         if ev:
             ev["t2"].record()
         if self.split_layout:
@@ -401,8 +406,9 @@ def measure(ep, wl, steps, warmup, rep, no_graph=False, sample_clocks=True):
         return [e[a].elapsed_time(e[b]) for e in evs]
 
     ops = {"layout": dict(stats_us(span("t0", "t1")),
-                          what="whole layout" if not wl.split_layout else "receive-row half (critical path)"),
-           "dispatch": dict(stats_us(span("t1", "t2")), bytes=alg["dispatch"]),
+                          what="layout and dispatch in one launch (ep_layout_dispatch)" if wl.fused else
+                          "whole layout" if not wl.split_layout else "receive-row half (critical path)"),
+           "dispatch": dict(stats_us(span("t0", "t2") if wl.fused else span("t1", "t2")), bytes=alg["dispatch"]),
            "combine": dict(stats_us(span("t3", "t4")), bytes=alg["combine"])}
     if wl.split_layout:
         ops["layout_pair_half"] = dict(stats_us(span("p0", "p1")), what="ep_layout_pairs on the side stream, beside dispatch")
@@ -416,7 +422,8 @@ def measure(ep, wl, steps, warmup, rep, no_graph=False, sample_clocks=True):
         ops["note"] = "per-kernel figures come from direct launches after a flush and include launch latency"
     return {"total_ms": total_ms, "step": stats_us(step_ms), "ops": ops, "launches": int(launches),
             "n_recv": n_recv, "n_pairs": n_pairs, "alg": alg, "launch": launch_note,
-            "layout": "one ep_layout call" if not wl.split_layout else
+            "layout": "ep_layout_dispatch (layout and dispatch in one launch)" if wl.fused else
+            "one ep_layout call" if not wl.split_layout else
             "ep_layout_ranks before dispatch, ep_layout_pairs on a side stream beside dispatch",
             "clocks": clocks.summary() if clocks else None}
 
@@ -659,6 +666,8 @@ def main():
     ap.add_argument("--no-graph", action="store_true", help="small workloads: time direct launches, not graph replays")
     ap.add_argument("--serial-layout", action="store_true",
                     help="one ep_layout call instead of the receive-row half before dispatch and the pair half beside it")
+    ap.add_argument("--separate-calls", action="store_true",
+                    help="small batches: ep_layout and ep_dispatch as two calls instead of ep_layout_dispatch")
     ap.add_argument("--variants", action="store_true",
                     help="also time the variants around the path (grouping, partial-output combine, dense baseline)")
     ap.add_argument("--no-configs", action="store_true", help="skip the extra configurations under `configs`")
@@ -686,7 +695,8 @@ def main():
     rcfg = inputs.shard_config(cfg, rank)            # replica `rank`: same shapes, its own seed stream
     T, K, H, E, R = cfg.T, cfg.K, cfg.H, cfg.E, cfg.R
 
-    wl = Workload(ep, inputs, cfg, rcfg, dev, args.seed, serial_layout=args.serial_layout)
+    wl = Workload(ep, inputs, cfg, rcfg, dev, args.seed, serial_layout=args.serial_layout,
+                  separate_calls=args.separate_calls)
     m = measure(ep, wl, args.steps, args.warmup, rep, no_graph=args.no_graph)
     n_recv, n_pairs, alg = m["n_recv"], m["n_pairs"], m["alg"]
     value = world * T * args.steps / (m["total_ms"] * 1e-3)

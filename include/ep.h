@@ -170,6 +170,23 @@ int ep_dispatch(const ep_shape_t *shape, const void *x, const int32_t *recv_slot
                 int64_t recv_capacity_rows, int32_t *status, void *stream);
 
 /*
+ * Layout and dispatch in one call (Section 4.5: at decode sizes the transfers are
+ * a few kilobytes and the cost is latency and synchronisation, not bytes; the
+ * routing-metadata step is what made routing-aware transfers slow). Produces
+ * exactly what ep_layout followed by ep_dispatch (with status = out->status)
+ * produces: every array of `out`, the dispatched rows in recv, and the status
+ * word (EP_STATUS_BAD_INDEX, EP_STATUS_CAPACITY when N_recv exceeds
+ * recv_capacity_rows). Batches of up to 1024 tokens whose routing table fits in
+ * shared memory take one launch in which every CTA derives the layout for itself
+ * and moves its own tokens' rows; larger batches run the two calls one after the
+ * other. Arguments as for ep_layout and ep_dispatch; the workspace is only used
+ * by the larger batches.
+ */
+int ep_layout_dispatch(const ep_shape_t *shape, const int32_t *topk_idx, const void *x, const ep_layout_t *out,
+                       void *workspace, size_t workspace_bytes, void *recv, int64_t recv_capacity_rows,
+                       void *stream);
+
+/*
  * Combine (Section 1; Section 4.3: the contributions that arrive for a token are
  * added on an SM): y[t][h] = bf16( sum_k w[t][k] * out[slot[t][k]][h] ), an fp32
  * fused multiply-add chain from +0 in ascending k, pairs with slot -1 skipped,

@@ -41,6 +41,9 @@ combine_rows_kernel(const uint4 *__restrict__ out, long long out_rows, const int
     const int lane = threadIdx.x & 31;
     const int g = threadIdx.x % G;
     const int t = blockIdx.x * (kBlock / G) + threadIdx.x / G;
+    // launched with programmatic stream serialisation: the CTAs may be resident before the previous
+    // kernel of the stream has finished; nothing is read or written before this returns
+    pdl_wait();
     if (t >= T) return;                                   // whole warps leave together (G >= 32)
 
     int32_t my_slot = -1;
@@ -155,12 +158,15 @@ int launch_combine(const ep_shape_t &s, const void *out, int64_t out_rows, const
     const uint4 *o = static_cast<const uint4 *>(out);
     uint4 *yd = static_cast<uint4 *>(y);
     const int G = vpr <= 64 ? 32 : (vpr <= 256 ? 64 : 128);
+    const long long rows = out_rows;
+    cudaError_t e;
     if (G == 32)
-        combine_rows_kernel<32><<<ceil_div(T, kBlock / 32), kBlock, 0, stream>>>(o, out_rows, slot, weights, yd, T, K, vpr, status);
+        e = launch_pdl(combine_rows_kernel<32>, dim3(ceil_div(T, kBlock / 32)), dim3(kBlock), 0, stream, o, rows, slot, weights, yd, T, K, vpr, status);
     else if (G == 64)
-        combine_rows_kernel<64><<<ceil_div(T, kBlock / 64), kBlock, 0, stream>>>(o, out_rows, slot, weights, yd, T, K, vpr, status);
+        e = launch_pdl(combine_rows_kernel<64>, dim3(ceil_div(T, kBlock / 64)), dim3(kBlock), 0, stream, o, rows, slot, weights, yd, T, K, vpr, status);
     else
-        combine_rows_kernel<128><<<T, kBlock, 0, stream>>>(o, out_rows, slot, weights, yd, T, K, vpr, status);
+        e = launch_pdl(combine_rows_kernel<128>, dim3(T), dim3(kBlock), 0, stream, o, rows, slot, weights, yd, T, K, vpr, status);
+    EP_CUDA_TRY(e);
     EP_LAUNCH_CHECK(1);
     return EP_OK;
 }

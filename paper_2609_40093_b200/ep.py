@@ -23,7 +23,7 @@ PROBE_READ, PROBE_WRITE, PROBE_COPY, PROBE_MEMCPY = 0, 1, 2, 3
 HOST_DUPLEX, HOST_PER_PEER, HOST_LOCAL_ON_DEVICE = 1, 2, 4
 
 EXPORTS = [
-    "ep_layout_workspace_bytes", "ep_layout", "ep_layout_ranks", "ep_layout_pairs", "ep_layout_static", "ep_layout_static_scratch_bytes", "ep_dispatch", "ep_combine", "ep_group",
+    "ep_layout_workspace_bytes", "ep_layout", "ep_layout_ranks", "ep_layout_pairs", "ep_layout_static", "ep_layout_static_scratch_bytes", "ep_layout_dispatch", "ep_dispatch", "ep_combine", "ep_group",
     "ep_combine_partial", "ep_dense_allgather", "ep_dense_reduce_scatter",
     "ep_host_roundtrip", "ep_host_dispatch_per_sender", "ep_host_combine", "ep_wait_senders", "ep_post_flags", "ep_host_step_pipelined",
     "ep_dispatch_copy_engine", "ep_host_step_arena_bytes", "ep_host_step", "ep_status",
@@ -72,6 +72,8 @@ def lib() -> ctypes.CDLL:
         L.ep_layout_static.restype = i32
         L.ep_layout_static_scratch_bytes.restype = sz
         L.ep_dispatch.argtypes = [sp, vp, vp, vp, i64, vp, vp]
+        L.ep_layout_dispatch.argtypes = [sp, vp, vp, ctypes.POINTER(_Layout), vp, sz, vp, i64, vp]
+        L.ep_layout_dispatch.restype = i32
         L.ep_combine.argtypes = [sp, vp, i64, vp, vp, vp, vp, vp]
         L.ep_group.argtypes = [sp, vp, i64, vp, vp, vp, i64, vp, vp]
         L.ep_combine_partial.argtypes = [sp, vp, i64, vp, vp, vp, vp, i64, vp, vp, vp]
@@ -212,6 +214,18 @@ def ep_layout_static(topk_idx: torch.Tensor, E: int, R: int, out: Layout) -> Lay
 
 def ep_layout_static_scratch_bytes() -> int:
     return int(lib().ep_layout_static_scratch_bytes())
+
+
+def ep_layout_dispatch(topk_idx: torch.Tensor, x: torch.Tensor, recv: torch.Tensor, E: int, R: int, out: Layout,
+                       workspace: torch.Tensor) -> Layout:
+    """`ep_layout` followed by `ep_dispatch`, one launch for batches of up to 1024 tokens."""
+    _want(topk_idx, torch.int32, "topk_idx"), _want(x, torch.bfloat16, "x"), _want(recv, torch.bfloat16, "recv")
+    T, K = topk_idx.shape
+    st = out.as_struct()
+    _check(lib().ep_layout_dispatch(ctypes.byref(_shape(T, K, x.shape[1], E, R)), _ptr(topk_idx), _ptr(x), ctypes.byref(st),
+                                    _ptr(workspace), workspace.numel(), _ptr(recv), recv.shape[0], _stream()),
+           "ep_layout_dispatch")
+    return out
 
 
 def ep_dispatch(x: torch.Tensor, recv_slot: torch.Tensor, recv: torch.Tensor, E: int, R: int, status=None):

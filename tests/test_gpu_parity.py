@@ -395,3 +395,89 @@ def test_largest_config_in_full():
     cfg = inputs.CONFIGS["C4"]
     d = inputs.make_inputs(cfg)
     _full_path_check(cfg, d["topk_idx"], d["topk_weights"], d["x"])
+
+
+FUSED = [  # T, H, E, K, R, routing: batches that take the one-launch layout + dispatch, and two that do not
+    (64, 256, 8, 2, 2, "uniform"),         # C1
+    (256, 4096, 8, 2, 8, "uniform"),       # C2
+    (1, 8, 1, 1, 1, "uniform"),
+    (2, 16, 2, 1, 2, "uniform"),
+    (8, 264, 8, 2, 4, "uniform"),
+    (96, 2880, 32, 4, 4, "uniform"),
+    (40, 520, 16, 4, 1, "uniform"),        # R = 1, 40 tokens: a ragged last group
+    (48, 72, 16, 3, 16, "uniform"),
+    (1000, 136, 512, 10, 8, "zipf"),
+    (1024, 7168, 256, 8, 8, "burst"),      # the largest fused batch, long rows
+    (320, 64, 4096, 4, 64, "uniform"),     # E and R at their maxima
+    (64, 64, 64, 32, 32, "uniform"),       # K at its maximum
+    (1023 - 1023 % 3, 40, 24, 5, 3, "zipf_identity"),
+    (1088, 64, 4096, 32, 64, "uniform"),   # does not fit: falls back to the two calls
+    (2048, 24, 128, 6, 8, "zipf"),         # more than 1024 tokens: falls back
+]
+
+
+@pytest.mark.parametrize("T,H,E,K,R,routing", FUSED)
+def test_layout_and_dispatch_in_one_call(T, H, E, K, R, routing):
+    cfg = inputs.custom_config(T, H, E, K, R, routing=routing, config_id=64)
+    d = inputs.make_inputs(cfg)
+    idx, x = d["topk_idx"].copy(), d["x"]
+    if T >= 8:                                             # masked, repeated and out-of-range ids
+        idx[1, :] = -1
+        idx[2, 0] = -1
+        idx[3, K - 1] = idx[3, 0]
+        idx[5, 0] = E + 3
+    ref = oracle.layout(idx, E, R)
+    lay = ep.alloc_layout(T, K, E, R, fill=-7)
+    ws = torch.empty(max(16, ep.ep_layout_workspace_bytes(T, K, E, R)), dtype=torch.uint8, device="cuda")
+    spare = 3
+    whole, recv = guarded(ref.n_recv + spare, H)
+    ep.ep_layout_dispatch(torch.from_numpy(idx).cuda(), dev_bf16(x), recv, E, R, lay, ws)
+    assert_layout_equal(lay, ref)
+    assert ep.ep_status(lay.status) == ref.status
+    np.testing.assert_array_equal(host_bits(recv), oracle.dispatch(x, ref.recv_slot, ref.n_recv + spare, fill=SENTINEL))
+    assert guards_intact(whole)
+    # a receive buffer that is too small: rows beyond it are skipped, the status says so
+    if ref.n_recv > 4:
+        cap = ref.n_recv - 3
+        whole, recv = guarded(cap, H)
+        ep.ep_layout_dispatch(torch.from_numpy(idx).cuda(), dev_bf16(x), recv, E, R, lay, ws)
+        assert ep.ep_status(lay.status) == ref.status | ep.STATUS_CAPACITY
+        np.testing.assert_array_equal(host_bits(recv), oracle.dispatch(x, ref.recv_slot, ref.n_recv)[:cap])
+        assert guards_intact(whole)
+
+
+def test_small_step_with_the_fused_call_replays_from_a_cuda_graph():
+    """layout+dispatch in one launch, combine launched with programmatic stream serialisation behind it:
+    captured once, replayed on new inputs."""
+    cfg = inputs.CONFIGS["C2"]
+    T, K, H, E, R = cfg.T, cfg.K, cfg.H, cfg.E, cfg.R
+    idx_d = torch.zeros(T, K, dtype=torch.int32, device="cuda")
+    w_d = torch.zeros(T, K, dtype=torch.float32, device="cuda")
+    x_d = torch.zeros(T, H, dtype=torch.bfloat16, device="cuda")
+    lay = ep.alloc_layout(T, K, E, R)
+    ws = torch.empty(16, dtype=torch.uint8, device="cuda")
+    recv = torch.zeros(T * min(K, R), H, dtype=torch.bfloat16, device="cuda")
+    y = torch.zeros(T, H, dtype=torch.bfloat16, device="cuda")
+
+    def step():
+        ep.ep_layout_dispatch(idx_d, x_d, recv, E, R, lay, ws)
+        ep.ep_combine(recv, lay.recv_slot, w_d, y, E, R, status=lay.status)
+
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        step()
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        step()
+    for seed in (5, 6):
+        d = inputs.make_inputs(cfg, seed)
+        idx_d.copy_(torch.from_numpy(d["topk_idx"]))
+        w_d.copy_(torch.from_numpy(d["topk_weights"]))
+        x_d.copy_(dev_bf16(d["x"]))
+        graph.replay()
+        torch.cuda.synchronize()
+        ref = oracle.layout(d["topk_idx"], E, R)
+        want = oracle.combine_f32(oracle.dispatch(d["x"], ref.recv_slot, ref.n_recv), ref.recv_slot, d["topk_weights"])
+        np.testing.assert_array_equal(host_bits(y), want)
+        assert ep.ep_status(lay.status) == 0
