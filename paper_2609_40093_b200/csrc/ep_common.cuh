@@ -55,7 +55,7 @@ int launch_combine(const ep_shape_t &s, const void *out, int64_t out_rows, const
 int launch_permute(int hidden, const void *src, int64_t src_rows, const int32_t *src_slot, void *dst,
                    int64_t dst_rows, const int32_t *dst_slot, int64_t n, int32_t *status, cudaStream_t stream);
 int launch_partial_rows(const ep_shape_t &s, const void *out, int64_t out_rows, const int32_t *pair_slot,
-                        const int32_t *recv_slot, const float *weights, void *partial, int64_t partial_rows,
+                        const int32_t *key, int dense, const float *weights, void *partial, int64_t partial_rows,
                         int32_t *status, cudaStream_t stream);
 int launch_sum_partial_rows(int hidden, int top_k, const void *partial, int64_t partial_rows, const int32_t *slot,
                             void *y, int n_tokens, int32_t *status, cudaStream_t stream);

@@ -381,7 +381,7 @@ extern "C" int ep_host_combine(const ep_shape_t *shape, const void *out, int64_t
     rc = begin_round(ev, half_free_events, round, up, down);
     if (rc != EP_OK) return rc;
     // every expert rank sums what it computed for a token into one row: these rows are what travels
-    rc = launch_partial_rows(*shape, out, out_rows, pair_slot, recv_slot, topk_weights, partial_send,
+    rc = launch_partial_rows(*shape, out, out_rows, pair_slot, recv_slot, 0, topk_weights, partial_send,
                              partial_capacity_rows, status, up);
     if (rc != EP_OK) return rc;
 
