@@ -324,14 +324,134 @@ class Workload:
             ev["t4"].record()
 
     @staticmethod
-    def new_events():
-        return {k: torch.cuda.Event(enable_timing=True) for k in ["t0", "t1", "t2", "t3", "t4", "p0", "p1"]}
+    def new_events(external=False):
+        kw = {"external": True} if external else {}
+        return {k: torch.cuda.Event(enable_timing=True, **kw) for k in ["t0", "t1", "t2", "t3", "t4", "p0", "p1"]}
+
+
+def small_direct(ep, wl, steps, flusher, rep, clocks, launches0):
+    """Small workloads, direct launches: every step after an L2 flush, timed by its own event pair."""
+    s_ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+    e_ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
+    rep.barrier()
+    if clocks:
+        clocks.__enter__()
+    for i in range(steps):
+        flusher()
+        s_ev[i].record()
+        wl.step()
+        e_ev[i].record()
+    torch.cuda.synchronize()
+    if clocks:
+        clocks.__exit__()
+    rep.barrier()
+    launches = ep.ep_launch_count() - launches0
+    evs = [wl.new_events() for _ in range(min(steps, 50))]
+    for e in evs:
+        flusher()
+        wl.step(e)
+    torch.cuda.synchronize()
+    return [s.elapsed_time(e) for s, e in zip(s_ev, e_ev)], evs, launches, "direct launches"
+
+
+def small_in_graph(ep, wl, steps, flusher, rep, clocks, per_graph=10):
+    """Small workloads, the deployment form of a decode step: a CUDA graph holds `per_graph` repetitions
+    of [L2 flush, event, step, event]; the events are recorded inside the graph, so the times are device
+    times of the step's kernels with neither host launch cost nor the flush in them. Per-kernel figures
+    come from a second graph with events between the calls. Also measures the floor of this protocol:
+    the same bracket around one and around three kernels that do nothing."""
+    def ext():
+        return torch.cuda.Event(enable_timing=True, external=True)
+
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):                        # per-device set-up of the calls outside any capture
+        flusher()
+        wl.step()
+    torch.cuda.synchronize()
+    n0 = ep.ep_launch_count()
+    wl.step()
+    torch.cuda.synchronize()
+    per_step_launches = ep.ep_launch_count() - n0
+
+    def build(body, n):
+        pairs = [(ext(), ext()) for _ in range(n)]
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            for s, e in pairs:
+                flusher()
+                s.record()
+                body()
+                e.record()
+        return g, pairs
+
+    g_step, pairs = build(wl.step, per_graph)
+    ops_evs = [wl.new_events(external=True) for _ in range(per_graph)]
+    g_ops = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g_ops):
+        for e in ops_evs:
+            flusher()
+            wl.step(e)
+    tiny = torch.zeros(64, dtype=torch.int32, device=wl.dev)
+    g_one, p_one = build(lambda: ep.ep_post_flags(tiny, 0, 1, 1), per_graph)
+    g_three, p_three = build(lambda: [ep.ep_post_flags(tiny, 0, 1, 1) for _ in range(3)], per_graph)
+    for g in (g_step, g_ops, g_one, g_three):            # warm replays
+        g.replay()
+    torch.cuda.synchronize()
+    step_ms = []
+    rep.barrier()
+    if clocks:
+        clocks.__enter__()
+    while len(step_ms) < steps:
+        g_step.replay()
+        torch.cuda.synchronize()
+        step_ms += [s.elapsed_time(e) for s, e in pairs]
+    if clocks:
+        clocks.__exit__()
+    rep.barrier()
+    step_ms = step_ms[:steps]
+
+    evs = []                                              # event times, read out after each replay
+    for _ in range(max(1, min(steps, 50) // per_graph)):
+        g_ops.replay()
+        torch.cuda.synchronize()
+        for e in ops_evs:
+            evs.append(FrozenEvents({(a, b): e[a].elapsed_time(e[b]) for a, b in
+                                     [("t0", "t1"), ("t1", "t2"), ("t0", "t2"), ("t2", "t3"), ("t3", "t4"), ("t0", "t4")]}))
+    floor = {}
+    for name, (g, ps) in [("one_empty_kernel_us", (g_one, p_one)), ("three_empty_kernels_us", (g_three, p_three))]:
+        ts = []
+        for _ in range(3):
+            g.replay()
+            torch.cuda.synchronize()
+            ts += [s.elapsed_time(e) * 1e3 for s, e in ps]
+        floor[name] = float(np.median(ts))
+    floor["what"] = ("the same in-graph bracket [flush, event, kernels, event] around kernels that do nothing: after the "
+                     "flush every kernel starts with cold instruction and parameter fetches; the event timer ticks in ~2 us steps")
+    return step_ms, evs, steps * per_step_launches, f"CUDA graph of {per_graph} x [flush, event, step, event]", floor
+
+
+class FrozenEvents:
+    """Event-pair durations read out earlier, behind the interface `measure` uses for live events."""
+
+    def __init__(self, spans):
+        self.spans = spans
+
+    def __getitem__(self, name):
+        return _FrozenEvent(self, name)
+
+
+class _FrozenEvent:
+    def __init__(self, owner, name):
+        self.owner, self.name = owner, name
+
+    def elapsed_time(self, other):
+        return self.owner.spans[(self.name, other.name)]
 
 
 def measure(ep, wl, steps, warmup, rep, no_graph=False, sample_clocks=True):
     """Times `steps` steps of a workload. Big workloads: back to back, direct launches, per-kernel events
-    inside the timed region. Small workloads: every step after an L2 flush, timed by its own event pair,
-    the step a CUDA-graph replay; per-kernel figures from a separate pass of direct launches."""
+    inside the timed region. Small workloads: every step after an L2 flush, timed by its own event pair
+    recorded inside a CUDA graph (small_in_graph), or with direct launches (small_direct)."""
     cfg, lay = wl.cfg, wl.lay
     for _ in range(warmup):
         wl.step()
@@ -344,62 +464,43 @@ def measure(ep, wl, steps, warmup, rep, no_graph=False, sample_clocks=True):
     dev_index = torch.cuda.current_device()
     clocks = ClockSampler(dev_index) if sample_clocks else None
     if not small:
-        evs = [wl.new_events() for _ in range(steps)]
+        # pass A, the timed region: K steps back to back, one event before and one after
         start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         rep.barrier()
         if clocks:
             clocks.__enter__()
         start.record()
         for i in range(steps):
-            wl.step(evs[i])
+            wl.step()
         stop.record()
         torch.cuda.synchronize()
-        if clocks:
-            clocks.__exit__()
         rep.barrier()
         launches = ep.ep_launch_count() - launches0
         total_ms = rep.max_over_ranks(start.elapsed_time(stop))
-        step_ms = [e["t0"].elapsed_time(e["t4"]) for e in evs]
-        launch_note = "direct launches"
-    else:
-        flusher = L2Flush(wl.dev)
-        graph = None
-        if not no_graph:
-            side = torch.cuda.Stream()
-            with torch.cuda.stream(side):
-                wl.step()
-            torch.cuda.synchronize()
-            graph = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(graph):
-                wl.step()
-        s_ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
-        e_ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps)]
-        rep.barrier()
-        if clocks:
-            clocks.__enter__()
+        # pass B, the same K steps again with events between the calls: per-kernel durations (the seven event
+        # records per step cost a few microseconds of stream time, which is why they are kept out of pass A)
+        evs = [wl.new_events() for _ in range(steps)]
+        start_b, stop_b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        start_b.record()
         for i in range(steps):
-            flusher()
-            s_ev[i].record()
-            graph.replay() if graph is not None else wl.step()
-            e_ev[i].record()
+            wl.step(evs[i])
+        stop_b.record()
         torch.cuda.synchronize()
         if clocks:
             clocks.__exit__()
         rep.barrier()
-        launches = ep.ep_launch_count() - launches0
-        if graph is not None:          # replays launch the captured kernels without passing through the library
-            n0 = ep.ep_launch_count()
-            wl.step()
-            torch.cuda.synchronize()
-            launches = steps * (ep.ep_launch_count() - n0)
-        step_ms = [s.elapsed_time(e) for s, e in zip(s_ev, e_ev)]
+        step_ms = [e["t0"].elapsed_time(e["t4"]) for e in evs]
+        launch_note = (f"direct launches; value from {steps} steps with no events inside; per-kernel durations from the "
+                       f"same {steps} steps repeated with events between the calls "
+                       f"({start_b.elapsed_time(stop_b) / steps * 1e3:.1f} us per step)")
+    else:
+        flusher = L2Flush(wl.dev)
+        floor = None
+        if no_graph:
+            step_ms, evs, launches, launch_note = small_direct(ep, wl, steps, flusher, rep, clocks, launches0)
+        else:
+            step_ms, evs, launches, launch_note, floor = small_in_graph(ep, wl, steps, flusher, rep, clocks)
         total_ms = rep.max_over_ranks(sum(step_ms))
-        evs = [wl.new_events() for _ in range(min(steps, 50))]
-        for e in evs:                  # per-kernel figures: direct launches, each step after a flush
-            flusher()
-            wl.step(e)
-        torch.cuda.synchronize()
-        launch_note = "CUDA graph replay of one step" if graph is not None else "direct launches"
         del flusher
 
     def span(a, b):
@@ -419,13 +520,59 @@ def measure(ep, wl, steps, warmup, rep, no_graph=False, sample_clocks=True):
         o["best_GB/s"] = o["bytes"] / (o["best_us"] * 1e-6) / 1e9
         o["tokens/s"] = cfg.T / (o["us"] * 1e-6)
     if small:
-        ops["note"] = "per-kernel figures come from direct launches after a flush and include launch latency"
-    return {"total_ms": total_ms, "step": stats_us(step_ms), "ops": ops, "launches": int(launches),
+        ops["note"] = ("per-kernel figures: events between the calls of a step" +
+                       (", direct launches after a flush (launch latency included)" if no_graph else
+                        " inside a graph, each step after a flush"))
+    return {"total_ms": total_ms, "step": stats_us(step_ms), "ops": ops, "launches": int(launches), "floor": floor if small else None,
             "n_recv": n_recv, "n_pairs": n_pairs, "alg": alg, "launch": launch_note,
             "layout": "ep_layout_dispatch (layout and dispatch in one launch)" if wl.fused else
             "one ep_layout call" if not wl.split_layout else
             "ep_layout_ranks before dispatch, ep_layout_pairs on a side stream beside dispatch",
             "clocks": clocks.summary() if clocks else None}
+
+
+def ops_alone(ep, wl, alg, per_graph=8, replays=4):
+    """Each call of the step by itself: [L2 flush, event, call, event] recorded inside a CUDA graph, so that a
+    kernel is charged neither launch latency nor the write-back of the previous kernel's dirty L2 lines (inside
+    the step, combine pays for up to ~60 MB of dispatch's output still sitting in L2)."""
+    cfg, lay = wl.cfg, wl.lay
+    E, R = cfg.E, cfg.R
+    flusher = L2Flush(wl.dev)
+    calls = {"layout": lambda: ep.ep_layout(wl.idx, E, R, out=lay, workspace=wl.ws),
+             "dispatch": lambda: ep.ep_dispatch(wl.x, lay.recv_slot, wl.recv, E, R, status=lay.status),
+             "combine": lambda: ep.ep_combine(wl.out, lay.pair_slot, wl.w, wl.y, E, R, status=lay.status)}
+    if wl.split_layout:
+        calls["layout_receive_row_half"] = lambda: ep.ep_layout_ranks(wl.idx, E, R, lay, wl.ws)
+    if wl.fused:
+        calls["layout_dispatch_one_launch"] = lambda: ep.ep_layout_dispatch(wl.idx, wl.x, wl.recv, E, R, lay, wl.ws)
+    res = {}
+    side = torch.cuda.Stream()
+    for name, fn in calls.items():
+        with torch.cuda.stream(side):
+            fn()
+        torch.cuda.synchronize()
+        pairs = [(torch.cuda.Event(enable_timing=True, external=True), torch.cuda.Event(enable_timing=True, external=True))
+                 for _ in range(per_graph)]
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            for s_, e_ in pairs:
+                flusher()
+                s_.record()
+                fn()
+                e_.record()
+        ts = []
+        for i in range(replays + 1):
+            g.replay()
+            torch.cuda.synchronize()
+            if i:
+                ts += [s_.elapsed_time(e_) for s_, e_ in pairs]
+        o = stats_us(ts)
+        if name in ("dispatch", "combine"):
+            o["GB/s"] = alg[name] / (o["us"] * 1e-6) / 1e9
+        res[name] = o
+        del g
+    del flusher
+    return res
 
 
 def time_variants(ep, wl, n_recv, n_pairs, iters=20):
@@ -638,6 +785,8 @@ def summarize_config(cfg, m, peak, host=None):
     ops = m["ops"]
     e = {"workload": workload_text(cfg), "step": m["step"], "tokens/s": cfg.T / (m["step"]["us"] * 1e-6),
          "launch": m["launch"], "layout_call": m["layout"], "n_recv": m["n_recv"], "n_pairs": m["n_pairs"], "ops": ops}
+    if m.get("floor"):
+        e["floor"] = m["floor"]
     for name in ("dispatch", "combine"):
         ops[name]["frac_of_measured_peak"] = ops[name]["GB/s"] / peak
         ops[name]["frac_of_nominal_8000"] = ops[name]["GB/s"] / NOMINAL_HBM_GBS
@@ -701,6 +850,7 @@ def main():
     n_recv, n_pairs, alg = m["n_recv"], m["n_pairs"], m["alg"]
     value = world * T * args.steps / (m["total_ms"] * 1e-3)
 
+    alone = ops_alone(ep, wl, alg) if not cfg.host_staged else None
     host = host_staged_arms(ep, wl) if cfg.host_staged else None
     variants = time_variants(ep, wl, n_recv, n_pairs) if args.variants else None
 
@@ -759,6 +909,11 @@ def main():
             m2 = measure(ep, w2, args.config_steps, max(5, args.warmup), rep, sample_clocks=False)
             h2 = host_staged_arms(ep, w2, iters=6, sweep=False) if c.host_staged else None
             configs[name] = summarize_config(c, m2, peak, h2)
+            if not c.host_staged:
+                al = ops_alone(ep, w2, m2["alg"])
+                for op in ("dispatch", "combine"):
+                    al[op]["frac_of_measured_peak"] = al[op]["GB/s"] / peak
+                configs[name]["ops_alone"] = al
             del w2
             torch.cuda.empty_cache()
 
@@ -772,8 +927,9 @@ def main():
         "warmup": args.warmup, "ms_per_step": m["total_ms"] / args.steps, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": config_object(cfg, world, n_recv, n_pairs),
-        "protocol": {"launch": m["launch"], "layout": m["layout"], "step": m["step"]},
+        "protocol": {"launch": m["launch"], "layout": m["layout"], "step": m["step"], "floor": m["floor"]},
         "ops": ops,
+        "ops_alone": alone,
         "roofline": roofline_object(cfg, "combine_rows_kernel", com_gbs, peak, peak_kind, probes),
         "roofline_dispatch": roofline_object(cfg, "dispatch_rows_kernel", dis_gbs, peak, peak_kind, probes),
         "probes": probes,
