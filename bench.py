@@ -260,7 +260,7 @@ def run_reference(args, cfg):
 class Workload:
     """Device buffers and the step of one configuration."""
 
-    def __init__(self, ep, inputs, cfg, rcfg, dev, seed, serial_layout=False, separate_calls=False):
+    def __init__(self, ep, inputs, cfg, rcfg, dev, seed, serial_layout=False, separate_calls=False, one_call=False):
         self.ep, self.cfg, self.dev = ep, cfg, dev
         T, K, H, E, R = cfg.T, cfg.K, cfg.H, cfg.E, cfg.R
         d = inputs.make_inputs(rcfg, seed)
@@ -285,6 +285,9 @@ class Workload:
         self.fork_ev, self.join_ev = torch.cuda.Event(), torch.cuda.Event()
         # decode-size batches: layout and dispatch in one launch (ep_layout_dispatch)
         self.fused = (not separate_calls) and T <= 1024 and not cfg.host_staged
+        self.one_call = one_call and not self.fused and not cfg.host_staged
+        if self.one_call:
+            self.split_layout = False
 
     def step(self, ev=None):
         """layout -> dispatch -> combine. Dispatch needs only the receive-row half of the layout, so for big
@@ -295,8 +298,8 @@ class Workload:
         main = torch.cuda.current_stream()
         if ev:
             ev["t0"].record()
-        if self.fused:
-            ep.ep_layout_dispatch(self.idx, self.x, self.recv, E, R, lay, self.ws)    # one launch for both
+        if self.fused or self.one_call:
+            ep.ep_layout_dispatch(self.idx, self.x, self.recv, E, R, lay, self.ws)    # small batches: one launch for both
         elif not self.split_layout:
             ep.ep_layout(self.idx, E, R, out=lay, workspace=self.ws)
         else:
@@ -311,7 +314,7 @@ class Workload:
             self.join_ev.record(self.side)
         if ev:
             ev["t1"].record()
-        if not self.fused:
+        if not (self.fused or self.one_call):
             ep.ep_dispatch(self.x, lay.recv_slot, self.recv, E, R, status=lay.status)
         if ev:
             ev["t2"].record()
@@ -817,6 +820,9 @@ def main():
                     help="one ep_layout call instead of the receive-row half before dispatch and the pair half beside it")
     ap.add_argument("--separate-calls", action="store_true",
                     help="small batches: ep_layout and ep_dispatch as two calls instead of ep_layout_dispatch")
+    ap.add_argument("--one-call", action="store_true",
+                    help="big batches: ep_layout_dispatch (whole layout, dispatch launched behind it with programmatic "
+                         "stream serialisation) instead of the split layout")
     ap.add_argument("--variants", action="store_true",
                     help="also time the variants around the path (grouping, partial-output combine, dense baseline)")
     ap.add_argument("--no-configs", action="store_true", help="skip the extra configurations under `configs`")
@@ -845,7 +851,7 @@ def main():
     T, K, H, E, R = cfg.T, cfg.K, cfg.H, cfg.E, cfg.R
 
     wl = Workload(ep, inputs, cfg, rcfg, dev, args.seed, serial_layout=args.serial_layout,
-                  separate_calls=args.separate_calls)
+                  separate_calls=args.separate_calls, one_call=args.one_call)
     m = measure(ep, wl, args.steps, args.warmup, rep, no_graph=args.no_graph)
     n_recv, n_pairs, alg = m["n_recv"], m["n_pairs"], m["alg"]
     value = world * T * args.steps / (m["total_ms"] * 1e-3)

@@ -46,7 +46,7 @@ int order_events(cudaEvent_t **pool, int need, std::unique_lock<std::mutex> &hol
 
 // Kernel launchers shared between the translation units (arguments already validated).
 int launch_dispatch(const ep_shape_t &s, const void *x, const int32_t *recv_slot, void *recv,
-                    int64_t capacity_rows, int32_t *status, cudaStream_t stream);
+                    int64_t capacity_rows, int32_t *status, cudaStream_t stream, bool behind_layout = false);
 int launch_group(const ep_shape_t &s, const void *recv, int64_t recv_rows, const int32_t *pair_row,
                  const int32_t *n_pairs, void *grouped, int64_t capacity_rows, int32_t *status,
                  cudaStream_t stream);
@@ -76,12 +76,12 @@ inline int check_shape(const ep_shape_t *s, bool need_hidden)
 
 inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 
-// Launch with programmatic stream serialisation: the kernel's CTAs may become resident while the
-// previous kernel of the stream is still running; the kernel must execute pdl_wait() before it
-// touches anything an earlier kernel wrote. Stream order is otherwise unchanged.
+// Launch through cudaLaunchKernelEx. pdl: with programmatic stream serialisation, i.e. the kernel's CTAs
+// may become resident while the previous kernel of the stream is still running; the kernel must execute
+// pdl_wait() before it touches anything an earlier kernel wrote. Stream order is otherwise unchanged.
 template <typename... KArgs, typename... Args>
-inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
-                              Args... args)
+inline cudaError_t launch_kernel(bool pdl, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                                 cudaStream_t stream, Args... args)
 {
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = grid;
@@ -92,8 +92,14 @@ inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, s
     attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr.val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = &attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = pdl ? 1 : 0;
     return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t stream,
+                              Args... args)
+{
+    return launch_kernel(true, kernel, grid, block, smem, stream, args...);
 }
 
 // --- device side ----------------------------------------------------------

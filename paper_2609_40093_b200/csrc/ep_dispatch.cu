@@ -48,8 +48,10 @@ dispatch_rows_kernel(const uint4 *__restrict__ x, const int32_t *__restrict__ re
     const int t = blockIdx.x * (blockDim.x / G) + threadIdx.x / G;
     if (t >= T) return;                                   // whole warps leave together (G % 32 == 0)
 
-    // the slot load and the first row loads are independent: issue both before anything waits on either
-    int32_t slot = lane < K ? __ldg(recv_slot + (size_t)t * K + lane) : -1;
+    // The first row loads do not depend on the slots: they are issued first. When the kernel was launched
+    // with programmatic stream serialisation behind the layout (ep_layout_dispatch: x is an input of that
+    // call and complete before the layout starts), this is where it waits for the slots to exist; in an
+    // ordinary launch the wait returns at once.
     const uint4 *src = x + (size_t)t * vec_per_row;
     uint4 buf[U];
 #pragma unroll
@@ -57,6 +59,8 @@ dispatch_rows_kernel(const uint4 *__restrict__ x, const int32_t *__restrict__ re
         const int v = g + u * G;
         if (v < vec_per_row) buf[u] = ld_stream(src + v);
     }
+    pdl_wait();
+    int32_t slot = lane < K ? __ldg(recv_slot + (size_t)t * K + lane) : -1;
     if (slot >= capacity_rows) {
         flag_status(status, EP_STATUS_CAPACITY);
         slot = -1;
@@ -177,19 +181,24 @@ int launch_permute(int hidden, const void *src, int64_t src_rows, const int32_t 
 }
 
 int launch_dispatch(const ep_shape_t &s, const void *x, const int32_t *recv_slot, void *recv,
-                    int64_t capacity_rows, int32_t *status, cudaStream_t stream)
+                    int64_t capacity_rows, int32_t *status, cudaStream_t stream, bool behind_layout)
 {
     const int T = s.num_tokens, K = s.top_k, vpr = s.hidden / 8;
     const uint4 *xs = static_cast<const uint4 *>(x);
     uint4 *rd = static_cast<uint4 *>(recv);
     const RowPlan p = plan_rows(vpr);
     const int grid = ceil_div(T, p.rows_per_block);
+    // behind_layout: the CTAs may become resident (and load their rows) while the layout kernel still runs
+    const long long cap = capacity_rows;
+    const dim3 g3(grid), b3(p.block);
+    cudaError_t e;
     switch (p.U) {
-    case 1: dispatch_rows_kernel<1><<<grid, p.block, 0, stream>>>(xs, recv_slot, rd, T, K, vpr, p.G, capacity_rows, status); break;
-    case 2: dispatch_rows_kernel<2><<<grid, p.block, 0, stream>>>(xs, recv_slot, rd, T, K, vpr, p.G, capacity_rows, status); break;
-    case 4: dispatch_rows_kernel<4><<<grid, p.block, 0, stream>>>(xs, recv_slot, rd, T, K, vpr, p.G, capacity_rows, status); break;
-    default: dispatch_rows_kernel<8><<<grid, p.block, 0, stream>>>(xs, recv_slot, rd, T, K, vpr, p.G, capacity_rows, status);
+    case 1: e = launch_kernel(behind_layout, dispatch_rows_kernel<1>, g3, b3, 0, stream, xs, recv_slot, rd, T, K, vpr, p.G, cap, status); break;
+    case 2: e = launch_kernel(behind_layout, dispatch_rows_kernel<2>, g3, b3, 0, stream, xs, recv_slot, rd, T, K, vpr, p.G, cap, status); break;
+    case 4: e = launch_kernel(behind_layout, dispatch_rows_kernel<4>, g3, b3, 0, stream, xs, recv_slot, rd, T, K, vpr, p.G, cap, status); break;
+    default: e = launch_kernel(behind_layout, dispatch_rows_kernel<8>, g3, b3, 0, stream, xs, recv_slot, rd, T, K, vpr, p.G, cap, status);
     }
+    EP_CUDA_TRY(e);
     EP_LAUNCH_CHECK(1);
     return EP_OK;
 }

@@ -286,10 +286,17 @@ extern "C" int ep_layout_dispatch(const ep_shape_t *shape, const int32_t *topk_i
     int rc = check_shape(shape, true);
     if (rc != EP_OK) return rc;
     const FusedPlan plan = plan_fused(*shape);
-    if (!plan.ok) {                                       // larger batches: the two calls, one after the other
+    if (!plan.ok) {
+        // larger batches: the layout, then the dispatch kernel launched with programmatic stream serialisation,
+        // so that its CTAs load their rows of x (an input of this call, complete before the layout starts)
+        // while the layout still runs, and wait for the slots on the device
         rc = ep_layout(shape, topk_idx, out, workspace, workspace_bytes, stream_);
         if (rc != EP_OK) return rc;
-        return ep_dispatch(shape, x, out->recv_slot, recv, recv_capacity_rows, out->status, stream_);
+        if (shape->num_tokens == 0) return EP_OK;
+        if (!x || !recv) return EP_ERR_NULL;
+        if (!aligned16(x) || !aligned16(recv) || recv_capacity_rows < 0) return EP_ERR_INVALID_ARG;
+        return launch_dispatch(*shape, x, out->recv_slot, recv, recv_capacity_rows, out->status,
+                               static_cast<cudaStream_t>(stream_), true);
     }
     if (!out || !topk_idx || !x || !recv) return EP_ERR_NULL;
     if (!out->expert_counts || !out->expert_offsets || !out->rank_rows || !out->rank_row_offsets ||

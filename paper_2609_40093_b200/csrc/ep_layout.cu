@@ -224,6 +224,7 @@ __global__ void __launch_bounds__(kMaxWarps * 32) layout_cta_count_kernel(Layout
 // ---------------------------------------------------------------- main kernel
 __global__ void __launch_bounds__(kMaxWarpsSingle * 32) layout_assign_kernel(LayoutArgs a)
 {
+    pdl_trigger();     // a kernel launched behind this one with programmatic serialisation may become resident
     extern __shared__ int32_t smem[];
     const int warps = blockDim.x >> 5, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int pw = a.bins + kMaxRanks + 64 * a.Kp;
