@@ -76,3 +76,51 @@ def test_binding_refuses_to_run_without_the_library(monkeypatch, tmp_path):
     monkeypatch.setattr(ep, "_LIB_PATH", str(tmp_path / "absent.so"))
     with pytest.raises(RuntimeError, match="missing"):
         ep.lib()
+
+
+def test_host_staged_calls_check_their_segment_tables_before_touching_a_gpu():
+    """ep_host_combine / ep_host_dispatch_per_sender validate the host copy of src_row_offsets (rows abut,
+    segments run forwards, the end fits the buffers) and their flags before any CUDA call is made."""
+    import numpy as np
+    L = ep.lib()
+    R, T, K, H, E = 4, 64, 2, 64, 8
+    shape = ep._shape(T, K, H, E, R)
+    p = ctypes.c_void_p(256)                                  # never dereferenced: every case fails on the host
+    good = np.zeros((R, R + 1), dtype=np.int32)
+    rows = np.arange(R * R + 1, dtype=np.int32) * 3           # 3 rows per segment
+    for r in range(R):
+        good[r] = rows[r * R:r * R + R + 1]
+
+    def combine(so, cap=int(good[-1, -1]), flags=0, bounce=p):
+        return L.ep_host_combine(ctypes.byref(shape), p, 128, p, p, p, so.ctypes.data_as(ctypes.c_void_p), p, p, cap,
+                                 bounce, 0, p, flags, None, None, None, None)
+
+    def per_sender(so, cap=int(good[-1, -1]), flags=0, timeout=0, sender_flags=None):
+        return L.ep_host_dispatch_per_sender(ctypes.byref(shape), p, p, p, so.ctypes.data_as(ctypes.c_void_p), p, p, cap,
+                                             p, 0, p, 128, sender_flags, 1, timeout, None, None, flags, None, None,
+                                             None, None, None)
+
+    backwards = good.copy()
+    backwards[1, 2] = backwards[1, 1] - 1
+    gap = good.copy()
+    gap[2:] += 1                                              # rank 2 does not start where rank 1 ends
+    shifted = good + 1                                        # first row is not 0
+    for call in (combine, per_sender):
+        assert call(backwards) == -2 and call(gap) == -2 and call(shifted) == -2
+        assert call(good, cap=int(good[-1, -1]) - 1) == -3    # buffers one row short
+        assert call(good, flags=8) == -2                      # unknown flag bit
+    assert combine(good, bounce=None) == -1
+    assert per_sender(good, sender_flags=p, timeout=0) == -2                  # a flag wait needs a time limit ...
+    assert per_sender(good, sender_flags=p, timeout=3_000_000_000) == -2      # ... of at most two seconds
+    assert L.ep_layout_dispatch(ctypes.byref(ep._shape(T, K, 60, E, R)), p, p, None, p, 16, p, 8, None) == -2
+    assert L.ep_layout_dispatch(ctypes.byref(shape), None, p, None, p, 16, p, 8, None) == -1
+
+
+def test_workspace_sizes_follow_the_launch_plan():
+    """One CTA up to 1024 tokens (no scratch), then one row of E+R+1 counters per CTA, at most 128 CTAs."""
+    ws = ep.ep_layout_workspace_bytes
+    assert ws(64, 2, 8, 2) == 16 and ws(1024, 8, 256, 8) == 16
+    assert ws(2048, 8, 256, 8) == 8 * (256 + 8 + 1) * 4       # 8 CTAs of 8 warps
+    assert ws(8192, 8, 256, 8) == 32 * (256 + 8 + 1) * 4
+    assert ws(65536, 8, 256, 8) == 128 * (256 + 8 + 1) * 4    # 128 CTAs, two 32-token groups per warp
+    assert ws(32768, 2, 4096, 64) > ep.ep_layout_static_scratch_bytes()
