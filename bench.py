@@ -388,6 +388,13 @@ def small_in_graph(ep, wl, steps, flusher, rep, clocks, per_graph=10):
         return g, pairs
 
     g_step, pairs = build(wl.step, per_graph)
+    warm_pairs = [(ext(), ext()) for _ in range(per_graph)]     # the same steps with nothing evicted in between
+    g_warm = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g_warm):
+        for s, e in warm_pairs:
+            s.record()
+            wl.step()
+            e.record()
     ops_evs = [wl.new_events(external=True) for _ in range(per_graph)]
     g_ops = torch.cuda.CUDAGraph()
     with torch.cuda.graph(g_ops):
@@ -428,6 +435,14 @@ def small_in_graph(ep, wl, steps, flusher, rep, clocks, per_graph=10):
             torch.cuda.synchronize()
             ts += [s.elapsed_time(e) * 1e3 for s, e in ps]
         floor[name] = float(np.median(ts))
+    warm = []
+    for _ in range(4):
+        g_warm.replay()
+        torch.cuda.synchronize()
+        warm += [s.elapsed_time(e) for s, e in warm_pairs]
+    floor["step_without_flush"] = dict(stats_us(warm[per_graph:]),
+                                       what="the same step replayed with L2 left warm (code and batch resident, as in a "
+                                            "decode loop); not the protocol figure")
     floor["what"] = ("the same in-graph bracket [flush, event, kernels, event] around kernels that do nothing: after the "
                      "flush every kernel starts with cold instruction and parameter fetches; the event timer ticks in ~2 us steps")
     return step_ms, evs, steps * per_step_launches, f"CUDA graph of {per_graph} x [flush, event, step, event]", floor

@@ -199,20 +199,18 @@ __global__ void __launch_bounds__(kFusedThreads) layout_dispatch_small_kernel(Fu
         const int t = g0 * 32 + lane;
         const bool mine = t >= t0 && t < t_end;
         const int32_t *row_ids = ids_all + t * a.Kp;
-        unsigned long long seen = 0ull;
         for (int k = 0; k < a.K; ++k) {
             const int e = row_ids[k];
             int32_t row = -1;
             if (e >= 0 && e < a.E) {
                 const int r = sdiv(e, a.mul_El);
                 row = tot[a.E + r] - n_pairs + grp_before[r] + __popc(bal_all[g0 * a.R + r] & lt);
-                if (mine && !((seen >> r) & 1ull)) {
-                    a.out.recv_token[row] = t;
-                    seen |= 1ull << r;
-                }
             }
             rows_own[lane * a.Kp + k] = row;
         }
+        for (int r = 0; r < a.R; ++r)                     // receive row -> token: one coalesced store per rank
+            if (mine && ((bal_all[g0 * a.R + r] >> lane) & 1u))
+                a.out.recv_token[tot[a.E + r] - n_pairs + grp_before[r] + __popc(bal_all[g0 * a.R + r] & lt)] = t;
         __syncwarp();
         const int first_pair = (t0 & 31) * a.K, own_pairs = (t_end - t0) * a.K;
         int32_t *pair_slot = a.out.pair_slot + (size_t)t0 * a.K, *recv_slot = a.out.recv_slot + (size_t)t0 * a.K;

@@ -108,7 +108,7 @@ struct LayoutArgs {
     const int32_t *idx;
     ep_layout_t out;
     int32_t *cta_part;  // [n_ctas][bins], global form only
-    int T, K, Kp, E, R, Tr;
+    int T, top_k, E, num_ranks, Tr;
     uint32_t mul_El, mul_K;
     FastDiv by_Tr;
     int tile_tokens, n_tiles, bins, n_ctas, mode;
@@ -118,11 +118,13 @@ struct LayoutArgs {
 
 // The warp copies the expert ids of the 32 tokens [tb, tb+32) into ids[32][Kp] (coalesced, eight loads
 // per lane in flight before the first use); entries of tokens >= t1 become -1. Returns the number of live items.
+template <int KT>
 __device__ __forceinline__ int stage_group(const LayoutArgs &a, int32_t *ids, int tb, int t1, int lane)
 {
-    const int n_items = (min(t1, tb + 32) - tb) * a.K;
-    const int32_t *src = a.idx + (size_t)tb * a.K;
-    for (int base = lane; base < 32 * a.K; base += 256) {
+    const int K = KT ? KT : a.top_k, Kp = K | 1;
+    const int n_items = (min(t1, tb + 32) - tb) * K;
+    const int32_t *src = a.idx + (size_t)tb * K;
+    for (int base = lane; base < 32 * K; base += 256) {
         int32_t v[8];
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
@@ -132,9 +134,9 @@ __device__ __forceinline__ int stage_group(const LayoutArgs &a, int32_t *ids, in
 #pragma unroll
         for (int u = 0; u < 8; ++u) {
             const int i = base + 32 * u;
-            if (i < 32 * a.K) {
+            if (i < 32 * K) {
                 const int tok = sdiv(i, a.mul_K);
-                ids[tok * a.Kp + (i - tok * a.K)] = v[u];
+                ids[tok * Kp + (i - tok * K)] = v[u];
             }
         }
     }
@@ -143,18 +145,22 @@ __device__ __forceinline__ int stage_group(const LayoutArgs &a, int32_t *ids, in
 }
 
 // position in ids[] / rows[] of pair i (in (t,k) order) of the staged group
+template <int KT>
 __device__ __forceinline__ int pair_pos(const LayoutArgs &a, int i)
 {
+    const int K = KT ? KT : a.top_k, Kp = K | 1;
     const int tok = sdiv(i, a.mul_K);
-    return tok * a.Kp + (i - tok * a.K);
+    return tok * Kp + (i - tok * K);
 }
 
 // rank bitmask of the token this lane owns in the staged group; *bad counts ids outside [-1, E)
+template <int KT>
 __device__ __forceinline__ unsigned long long token_rank_mask(const LayoutArgs &a, const int32_t *ids, int lane, int *bad)
 {
+    const int K = KT ? KT : a.top_k, Kp = K | 1;
     unsigned long long mask = 0ull;
-    for (int k = 0; k < a.K; ++k) {
-        const int e = ids[lane * a.Kp + k];
+    for (int k = 0; k < K; ++k) {
+        const int e = ids[lane * Kp + k];
         if (e >= 0 && e < a.E) mask |= 1ull << sdiv(e, a.mul_El);
         else if (e != -1) ++*bad;
     }
@@ -164,9 +170,10 @@ __device__ __forceinline__ unsigned long long token_rank_mask(const LayoutArgs &
 // One warp counts its tile into hist[bins]. kShared == false: hist is this warp's own and is
 // zeroed here; kShared == true: hist is one histogram for the whole CTA, zeroed by the caller.
 // Returns the rank mask of this lane's token in the tile's last group (reused by a one-group replay).
-template <bool kShared>
+template <bool kShared, int KT, int RT>
 __device__ __forceinline__ unsigned long long count_tile(const LayoutArgs &a, int32_t *hist, int32_t *ids, int tile, int lane)
 {
+    const int K = KT ? KT : a.top_k, Kp = K | 1, R = RT ? RT : a.num_ranks;
     if (!kShared) {
         for (int b = a.blo + lane; b < a.bins; b += 32) hist[b] = 0;
         __syncwarp();
@@ -178,14 +185,14 @@ __device__ __forceinline__ unsigned long long count_tile(const LayoutArgs &a, in
     int hits0 = 0, hits1 = 0;                        // lane l counts the hits of ranks l and l + 32
     unsigned long long mask = 0ull;
     for (int tb = t0; tb < t1; tb += 32) {
-        stage_group(a, ids, tb, t1, lane);
+        stage_group<KT>(a, ids, tb, t1, lane);
         if (a.blo == 0)                               // experts: any order
-            for (int k = 0; k < a.K; ++k) {
-                const int e = ids[lane * a.Kp + k];
+            for (int k = 0; k < K; ++k) {
+                const int e = ids[lane * Kp + k];
                 if (e >= 0 && e < a.E) atomicAdd(hist + e, 1);
             }
-        mask = token_rank_mask(a, ids, lane, &bad);   // rank hits: token per lane, ballot per rank
-        for (int r = 0; r < a.R; ++r) {
+        mask = token_rank_mask<KT>(a, ids, lane, &bad);   // rank hits: token per lane, ballot per rank
+        for (int r = 0; r < R; ++r) {
             const int c = __popc(__ballot_sync(kFullMask, (mask >> r) & 1ull));
             if (lane == (r & 31)) {
                 if (r < 32) hits0 += c;
@@ -195,44 +202,48 @@ __device__ __forceinline__ unsigned long long count_tile(const LayoutArgs &a, in
         __syncwarp();
     }
     if (kShared) {
-        if (lane < a.R && hits0) atomicAdd(hist + a.E + lane, hits0);
-        if (lane + 32 < a.R && hits1) atomicAdd(hist + a.E + 32 + lane, hits1);
+        if (lane < R && hits0) atomicAdd(hist + a.E + lane, hits0);
+        if (lane + 32 < R && hits1) atomicAdd(hist + a.E + 32 + lane, hits1);
     } else {
-        if (lane < a.R) hist[a.E + lane] = hits0;
-        if (lane + 32 < a.R) hist[a.E + 32 + lane] = hits1;
+        if (lane < R) hist[a.E + lane] = hits0;
+        if (lane + 32 < R) hist[a.E + 32 + lane] = hits1;
     }
-    if (bad) atomicAdd(hist + a.E + a.R, bad);
+    if (bad) atomicAdd(hist + a.E + R, bad);
     __syncwarp();
     return mask;
 }
 
 // ---------------------------------------------------------------- global form, first kernel
+template <int KT, int RT>
 __global__ void __launch_bounds__(kMaxWarps * 32) layout_cta_count_kernel(LayoutArgs a)
 {
+    const int K = KT ? KT : a.top_k, Kp = K | 1;
     pdl_trigger();                                                    // the main kernel may start its own counting now
     extern __shared__ int32_t smem[];
     const int warps = blockDim.x >> 5, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     // one histogram for the CTA (first `bins` words), per-warp id staging behind it
     for (int b = a.blo + threadIdx.x; b < a.bins; b += blockDim.x) smem[b] = 0;
     __syncthreads();
-    count_tile<true>(a, smem, smem + a.bins + warp * 32 * a.Kp, blockIdx.x * warps + warp, lane);
+    count_tile<true, KT, RT>(a, smem, smem + a.bins + warp * 32 * Kp, blockIdx.x * warps + warp, lane);
     __syncthreads();
     int32_t *dst = a.cta_part + (size_t)blockIdx.x * a.bins;
     for (int b = a.blo + threadIdx.x; b < a.bins; b += blockDim.x) dst[b] = smem[b];
 }
 
 // ---------------------------------------------------------------- main kernel
+template <int KT, int RT>
 __global__ void __launch_bounds__(kMaxWarpsSingle * 32) layout_assign_kernel(LayoutArgs a)
 {
+    const int K = KT ? KT : a.top_k, Kp = K | 1, R = RT ? RT : a.num_ranks;
     pdl_trigger();     // a kernel launched behind this one with programmatic serialisation may become resident
     extern __shared__ int32_t smem[];
     const int warps = blockDim.x >> 5, warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int pw = a.bins + kMaxRanks + 64 * a.Kp;
-    const int nb = a.E + a.R;
+    const int pw = a.bins + kMaxRanks + 64 * Kp;
+    const int nb = a.E + R;
     int32_t *run = smem + warp * pw;                                 // [bins] histogram, later next free slot
     unsigned *bal = reinterpret_cast<unsigned *>(run + a.bins);      // [R] ballots of the current 32 tokens
     int32_t *rows = run + a.bins + kMaxRanks;                        // [32][Kp] receive rows of the current 32 tokens
-    int32_t *ids = rows + 32 * a.Kp;                                 // [32][Kp] expert ids of the current 32 tokens
+    int32_t *ids = rows + 32 * Kp;                                 // [32][Kp] expert ids of the current 32 tokens
     int32_t *tot = smem + warps * pw;                                // [E+R+1] totals -> one scan: experts, then ranks
     int32_t *pre = tot + a.bins + 1;                                 // [bins] count in earlier CTAs
     int32_t *cta_tot = pre + a.bins;                                 // [bins] this CTA's totals (peers read it)
@@ -240,7 +251,7 @@ __global__ void __launch_bounds__(kMaxWarpsSingle * 32) layout_assign_kernel(Lay
     const int tile = blockIdx.x * warps + warp;
     const unsigned lt = lanemask_lt();
 
-    const unsigned long long mask_kept = count_tile<false>(a, run, ids, tile, lane);
+    const unsigned long long mask_kept = count_tile<false, KT, RT>(a, run, ids, tile, lane);
     __syncthreads();
     const bool ranks = a.parts & kPartRanks, pairs = a.parts & kPartPairs;
     for (int b = a.blo + threadIdx.x; b < a.bins; b += blockDim.x) {  // this CTA's total per bin
@@ -290,9 +301,9 @@ __global__ void __launch_bounds__(kMaxWarpsSingle * 32) layout_assign_kernel(Lay
         if (pairs)
             for (int e = threadIdx.x; e <= a.E; e += blockDim.x) a.out.expert_offsets[e] = tot[e];
         if (ranks) {
-            for (int r = threadIdx.x; r <= a.R; r += blockDim.x) a.out.rank_row_offsets[r] = tot[a.E + r] - n_pairs;
-            for (int r = threadIdx.x; r < a.R; r += blockDim.x)
-                a.out.src_row_offsets[r * (a.R + 1) + a.R] = tot[a.E + r + 1] - n_pairs;
+            for (int r = threadIdx.x; r <= R; r += blockDim.x) a.out.rank_row_offsets[r] = tot[a.E + r] - n_pairs;
+            for (int r = threadIdx.x; r < R; r += blockDim.x)
+                a.out.src_row_offsets[r * (R + 1) + R] = tot[a.E + r + 1] - n_pairs;
         }
     }
     // next free slot of every bin for every warp: offset + earlier CTAs + earlier warps of this CTA
@@ -323,14 +334,14 @@ __global__ void __launch_bounds__(kMaxWarpsSingle * 32) layout_assign_kernel(Lay
         int n_items, bad = 0;
         unsigned long long mask;
         if (a.tile_tokens == 32) {
-            n_items = (min(t1, tb + 32) - tb) * a.K;
+            n_items = (min(t1, tb + 32) - tb) * K;
             mask = mask_kept;
         } else {
-            n_items = stage_group(a, ids, tb, t1, lane);
-            mask = token_rank_mask(a, ids, lane, &bad);
+            n_items = stage_group<KT>(a, ids, tb, t1, lane);
+            mask = token_rank_mask<KT>(a, ids, lane, &bad);
         }
         // --- receive rows: which of these 32 tokens hit which rank (lane r keeps rank r's ballot)
-        for (int r = 0; r < a.R; ++r) {
+        for (int r = 0; r < R; ++r) {
             const unsigned b = __ballot_sync(kFullMask, (mask >> r) & 1ull);
             if (lane == (r & 31)) bal[r] = b;
         }
@@ -338,34 +349,34 @@ __global__ void __launch_bounds__(kMaxWarpsSingle * 32) layout_assign_kernel(Lay
         if (live) {
             const int s = fdiv(t, a.by_Tr);
             if (ranks && t == s * a.Tr)              // first token of source rank s
-                for (int r = 0; r < a.R; ++r)
-                    a.out.src_row_offsets[r * (a.R + 1) + s] = run[a.E + r] + __popc(bal[r] & lt);
-            unsigned long long seen = 0ull;
-            for (int k = 0; k < a.K; ++k) {
-                const int e = ids[lane * a.Kp + k];
+                for (int r = 0; r < R; ++r)
+                    a.out.src_row_offsets[r * (R + 1) + s] = run[a.E + r] + __popc(bal[r] & lt);
+            for (int k = 0; k < K; ++k) {
+                const int e = ids[lane * Kp + k];
                 int32_t row = -1;
                 if (e >= 0 && e < a.E) {
                     const int r = sdiv(e, a.mul_El);
                     row = run[a.E + r] + __popc(bal[r] & lt);
-                    if (ranks && !((seen >> r) & 1ull)) {
-                        a.out.recv_token[row] = t;
-                        seen |= 1ull << r;
-                    }
                 }
-                rows[lane * a.Kp + k] = row;
+                rows[lane * Kp + k] = row;
             }
         }
+        // receive row -> token, rank by rank: the tokens of these 32 that hit rank r own consecutive rows, so
+        // each rank costs one store to one or two cache lines (a store per pick would touch a line per rank)
+        if (ranks)
+            for (int r = 0; r < R; ++r)
+                if (live && ((mask >> r) & 1ull)) a.out.recv_token[run[a.E + r] + __popc(bal[r] & lt)] = t;
         __syncwarp();
-        for (int r = lane; r < a.R; r += 32) run[a.E + r] += __popc(bal[r]);
+        for (int r = lane; r < R; r += 32) run[a.E + r] += __popc(bal[r]);
         __syncwarp();
-        int32_t *recv_slot = a.out.recv_slot + (size_t)tb * a.K;
+        int32_t *recv_slot = a.out.recv_slot + (size_t)tb * K;
         if (!pairs) {                                // receive-row half only: publish the rows and go on
-            for (int i = lane; i < n_items; i += 32) recv_slot[i] = rows[pair_pos(a, i)];
+            for (int i = lane; i < n_items; i += 32) recv_slot[i] = rows[pair_pos<KT>(a, i)];
             __syncwarp();
             continue;
         }
         // --- pair slots: the items of these tokens, 32 at a time in (t,k) order
-        int32_t *pair_slot = a.out.pair_slot + (size_t)tb * a.K;
+        int32_t *pair_slot = a.out.pair_slot + (size_t)tb * K;
         for (int j0 = 0; j0 < n_items; j0 += 32 * kSteps) {          // kSteps steps of 32 pairs: their matches, then their
             int pos[kSteps], e[kSteps], leader[kSteps];              // counter updates in order, then their stores
             unsigned m[kSteps];
@@ -374,7 +385,7 @@ __global__ void __launch_bounds__(kMaxWarpsSingle * 32) layout_assign_kernel(Lay
             for (int u = 0; u < kSteps; ++u) {
                 const int i = j0 + 32 * u + lane;
                 const int tok = sdiv(i, a.mul_K);
-                pos[u] = tok * a.Kp + (i - tok * a.K);
+                pos[u] = tok * Kp + (i - tok * K);
                 e[u] = i < n_items ? ids[pos[u]] : -1;
                 if (e[u] >= a.E) e[u] = -2;                          // out of range: masked like any negative id
             }
@@ -421,12 +432,36 @@ extern "C" size_t ep_layout_workspace_bytes(const ep_shape_t *shape)
 namespace ep {
 namespace {
 
+// The kernels are compiled for the common (top-k, ranks) pairs with both as compile-time constants (their
+// loops unroll: the receive-row half of T=8192, K=8, R=8 takes 7.7 us instead of 9.4) and once with both
+// read at run time.
+using LayoutKernel = void (*)(LayoutArgs);
+struct KernelPair {
+    LayoutKernel count, assign;
+};
+template <int KT, int RT>
+constexpr KernelPair kernel_pair() { return KernelPair{layout_cta_count_kernel<KT, RT>, layout_assign_kernel<KT, RT>}; }
+
+constexpr int kTunedTopK[] = {2, 4, 6, 8};
+constexpr int kTunedRanks = 8;
+constexpr int kNumKernelPairs = 5;
+const KernelPair kKernelPairs[kNumKernelPairs] = {kernel_pair<0, 0>(), kernel_pair<2, kTunedRanks>(), kernel_pair<4, kTunedRanks>(),
+                                                  kernel_pair<6, kTunedRanks>(), kernel_pair<8, kTunedRanks>()};
+
+int pick_kernels(int K, int R)
+{
+    if (R == kTunedRanks)
+        for (int i = 0; i < 4; ++i)
+            if (K == kTunedTopK[i]) return i + 1;
+    return 0;
+}
+
 // Can `cfg` (one cluster = the whole grid) be resident on device `dev`? Asked once per device and
 // (cluster size, CTA size, shared memory) and remembered; "no" sends the call to the global form.
-bool cluster_fits(int dev, const cudaLaunchConfig_t &cfg)
+bool cluster_fits(int dev, int which, const cudaLaunchConfig_t &cfg)
 {
     struct Key {
-        int dev;
+        int dev, which;
         unsigned ctas, threads;
         size_t smem;
         bool fits;
@@ -436,14 +471,14 @@ bool cluster_fits(int dev, const cudaLaunchConfig_t &cfg)
     static int n_known = 0;
     std::lock_guard<std::mutex> lock(mu);
     for (int i = 0; i < n_known; ++i)
-        if (known[i].dev == dev && known[i].ctas == cfg.gridDim.x && known[i].threads == cfg.blockDim.x &&
+        if (known[i].dev == dev && known[i].which == which && known[i].ctas == cfg.gridDim.x && known[i].threads == cfg.blockDim.x &&
             known[i].smem == cfg.dynamicSmemBytes)
             return known[i].fits;
     int n = 0;
-    const cudaError_t e = cudaOccupancyMaxActiveClusters(&n, layout_assign_kernel, &cfg);
+    const cudaError_t e = cudaOccupancyMaxActiveClusters(&n, kKernelPairs[which].assign, &cfg);
     if (e != cudaSuccess) (void)cudaGetLastError();         // treated as "does not fit"; not this call's error
     const bool fits = e == cudaSuccess && n >= 1;
-    if (n_known < 32) known[n_known++] = Key{dev, cfg.gridDim.x, cfg.blockDim.x, cfg.dynamicSmemBytes, fits};
+    if (n_known < 32) known[n_known++] = Key{dev, which, cfg.gridDim.x, cfg.blockDim.x, cfg.dynamicSmemBytes, fits};
     return fits;
 }
 
@@ -482,7 +517,7 @@ int run_layout(const ep_shape_t *shape, const int32_t *topk_idx, const ep_layout
     a.idx = topk_idx;
     a.out = *out;
     a.cta_part = static_cast<int32_t *>(workspace);
-    a.T = T; a.K = shape->top_k; a.Kp = shape->top_k | 1; a.E = E; a.R = R; a.Tr = T / R;
+    a.T = T; a.top_k = shape->top_k; a.E = E; a.num_ranks = R; a.Tr = T / R;
     a.mul_El = small_div_mul(E / R); a.mul_K = small_div_mul(shape->top_k); a.by_Tr = make_fastdiv(T / R);
     a.tile_tokens = plan.tile_tokens; a.n_tiles = plan.n_tiles; a.bins = plan.bins; a.n_ctas = plan.n_ctas;
     a.mode = plan.mode;
@@ -494,10 +529,13 @@ int run_layout(const ep_shape_t *shape, const int32_t *topk_idx, const ep_layout
     EP_CUDA_TRY(cudaGetDevice(&dev));
     if (dev < 0 || dev >= 64) return EP_ERR_INVALID_ARG;
     if (!attr_done[dev].load(std::memory_order_acquire)) {
-        EP_CUDA_TRY(cudaFuncSetAttribute(layout_cta_count_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget));
-        EP_CUDA_TRY(cudaFuncSetAttribute(layout_assign_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget));
+        for (int i = 0; i < kNumKernelPairs; ++i) {
+            EP_CUDA_TRY(cudaFuncSetAttribute(kKernelPairs[i].count, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget));
+            EP_CUDA_TRY(cudaFuncSetAttribute(kKernelPairs[i].assign, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget));
+        }
         attr_done[dev].store(true, std::memory_order_release);
     }
+    const int which = pick_kernels(shape->top_k, R);
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(plan.n_ctas);
     cfg.blockDim = dim3(plan.warps * 32);
@@ -512,14 +550,14 @@ int run_layout(const ep_shape_t *shape, const int32_t *topk_idx, const ep_layout
         attr.val.clusterDim.z = 1;
         cfg.attrs = &attr;
         cfg.numAttrs = 1;
-        if (!cluster_fits(dev, cfg)) {                      // this device cannot co-schedule the cluster
+        if (!cluster_fits(dev, which, cfg)) {                      // this device cannot co-schedule the cluster
             a.mode = kModeGlobal;
             cfg.attrs = nullptr;
             cfg.numAttrs = 0;
         }
     }
     if (a.mode == kModeGlobal) {
-        layout_cta_count_kernel<<<plan.n_ctas, plan.warps * 32, plan.smem, stream>>>(a);
+        kKernelPairs[which].count<<<plan.n_ctas, plan.warps * 32, plan.smem, stream>>>(a);
         // the main kernel may start while the first still runs; it waits on the device before it reads cta_part
         attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
         attr.val.programmaticStreamSerializationAllowed = 1;
@@ -527,7 +565,7 @@ int run_layout(const ep_shape_t *shape, const int32_t *topk_idx, const ep_layout
         cfg.numAttrs = 1;
         launched = 2;
     }
-    EP_CUDA_TRY(cudaLaunchKernelEx(&cfg, layout_assign_kernel, a));
+    EP_CUDA_TRY(cudaLaunchKernelEx(&cfg, kKernelPairs[which].assign, a));
     EP_LAUNCH_CHECK(launched);
     return EP_OK;
 }
