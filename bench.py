@@ -260,7 +260,7 @@ def run_reference(args, cfg):
 class Workload:
     """Device buffers and the step of one configuration."""
 
-    def __init__(self, ep, inputs, cfg, rcfg, dev, seed, serial_layout=False, separate_calls=False, one_call=False):
+    def __init__(self, ep, inputs, cfg, rcfg, dev, seed, serial_layout=False, separate_calls=False, one_call=False, force_split=False):
         self.ep, self.cfg, self.dev = ep, cfg, dev
         T, K, H, E, R = cfg.T, cfg.K, cfg.H, cfg.E, cfg.R
         d = inputs.make_inputs(rcfg, seed)
@@ -279,8 +279,8 @@ class Workload:
         else:
             self.recv = torch.empty(T * min(K, R), H, dtype=torch.bfloat16, device=dev)
         self.y = torch.empty(T, H, dtype=torch.bfloat16, device=dev)
-        # big batches: the pair half of the layout runs beside dispatch; launch-bound batches keep one call
-        self.split_layout = (not serial_layout) and not is_small(cfg) and not cfg.host_staged
+        # prefill-size batches (T >= 4096): the pair half of the layout runs beside dispatch; smaller ones keep one call
+        self.split_layout = (not serial_layout) and (T >= 4096 or force_split) and not cfg.host_staged
         self.side = torch.cuda.Stream()
         self.fork_ev, self.join_ev = torch.cuda.Event(), torch.cuda.Event()
         # decode-size batches: layout and dispatch in one launch (ep_layout_dispatch)
@@ -425,8 +425,10 @@ def small_in_graph(ep, wl, steps, flusher, rep, clocks, per_graph=10):
         g_ops.replay()
         torch.cuda.synchronize()
         for e in ops_evs:
-            evs.append(FrozenEvents({(a, b): e[a].elapsed_time(e[b]) for a, b in
-                                     [("t0", "t1"), ("t1", "t2"), ("t0", "t2"), ("t2", "t3"), ("t3", "t4"), ("t0", "t4")]}))
+            spans = [("t0", "t1"), ("t1", "t2"), ("t0", "t2"), ("t2", "t3"), ("t3", "t4"), ("t0", "t4")]
+            if wl.split_layout:
+                spans.append(("p0", "p1"))
+            evs.append(FrozenEvents({(a, b): e[a].elapsed_time(e[b]) for a, b in spans}))
     floor = {}
     for name, (g, ps) in [("one_empty_kernel_us", (g_one, p_one)), ("three_empty_kernels_us", (g_three, p_three))]:
         ts = []
@@ -835,6 +837,7 @@ def main():
                     help="one ep_layout call instead of the receive-row half before dispatch and the pair half beside it")
     ap.add_argument("--separate-calls", action="store_true",
                     help="small batches: ep_layout and ep_dispatch as two calls instead of ep_layout_dispatch")
+    ap.add_argument("--force-split", action="store_true", help="split layout (pair half on a side stream) also for small batches")
     ap.add_argument("--one-call", action="store_true",
                     help="big batches: ep_layout_dispatch (whole layout, dispatch launched behind it with programmatic "
                          "stream serialisation) instead of the split layout")
@@ -866,7 +869,7 @@ def main():
     T, K, H, E, R = cfg.T, cfg.K, cfg.H, cfg.E, cfg.R
 
     wl = Workload(ep, inputs, cfg, rcfg, dev, args.seed, serial_layout=args.serial_layout,
-                  separate_calls=args.separate_calls, one_call=args.one_call)
+                  separate_calls=args.separate_calls, one_call=args.one_call, force_split=args.force_split)
     m = measure(ep, wl, args.steps, args.warmup, rep, no_graph=args.no_graph)
     n_recv, n_pairs, alg = m["n_recv"], m["n_pairs"], m["alg"]
     value = world * T * args.steps / (m["total_ms"] * 1e-3)

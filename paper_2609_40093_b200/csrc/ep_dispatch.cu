@@ -46,6 +46,7 @@ dispatch_rows_kernel(const uint4 *__restrict__ x, const int32_t *__restrict__ re
     const int lane = threadIdx.x & 31;
     const int g = threadIdx.x % G;                       // position inside the row group
     const int t = blockIdx.x * (blockDim.x / G) + threadIdx.x / G;
+    pdl_trigger();     // a kernel launched behind this one with programmatic serialisation may become resident
     if (t >= T) return;                                   // whole warps leave together (G % 32 == 0)
 
     // The first row loads do not depend on the slots: they are issued first. When the kernel was launched
