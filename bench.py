@@ -34,7 +34,7 @@ UNIT = "tokens/s"
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes per launch of the dominant kernels from the committed ncu captures (profiles/).
-NCU_TRAFFIC_BYTES = {("C4", "combine_rows_kernel"): 1038.7e6, ("C4", "dispatch_rows_kernel"): 680.8e6}
+NCU_TRAFFIC_BYTES = {("C4", "combine_rows_kernel"): 1038.7e6, ("C4", "dispatch_rows_kernel"): 680.9e6}
 L2_BYTES = 126e6
 CONTEXT = ("paper reports 2.00x (dispatch) / 1.53x (combine) over NCCL for its dense all-gather/"
            "reduce-scatter on RTX 4090/5090 PCIe boxes; no number for the routing-aware path")
