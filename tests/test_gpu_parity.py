@@ -25,7 +25,9 @@ EDGE = [  # T, H, E, K, R, routing
     (40, 520, 16, 4, 1, "uniform"),        # R = 1
     (48, 72, 16, 3, 16, "uniform"),        # E = R
     (1000, 136, 512, 10, 8, "zipf"),       # 10 of 512, the finest model the paper names
-    (1088, 64, 4096, 32, 64, "uniform"),   # every maximum at once: K=32, E=4096, R=64
+    (1088, 64, 4096, 32, 64, "uniform"),   # every maximum at once: K=32, E=4096, R=64 (a 7-CTA cluster of 197 KB CTAs)
+    (320, 8, 4096, 32, 64, "uniform"),     # the same limits, two CTAs
+    (3200, 8, 4096, 32, 64, "uniform"),    # the same limits past the cluster: 17 CTAs, two kernels
     (40000, 8, 16, 2, 8, "uniform"),       # more than 1024*32 tokens: layout tiles of 64 tokens, 16-byte rows
     (33 * 8, 40, 24, 5, 8, "zipf_identity"),
     (65536, 8, 256, 8, 8, "burst"),        # 128 layout CTAs, tiles of 64 tokens, half a million pairs
