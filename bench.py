@@ -274,6 +274,7 @@ class Workload:
         self.lay = ep.alloc_layout(T, K, E, R, device=dev)
         self.ws = torch.empty(max(16, ep.ep_layout_workspace_bytes(T, K, E, R)), dtype=torch.uint8, device=dev)
         self.ws2 = torch.empty_like(self.ws)
+        self.ws_both = torch.empty(2 * self.ws.numel() + 256, dtype=torch.uint8, device=dev)
         if cfg.host_staged:
             self.recv = torch.empty(T * min(K, R), H, dtype=torch.bfloat16).pin_memory()
         else:
@@ -283,11 +284,15 @@ class Workload:
         self.split_layout = (not serial_layout) and (T >= 4096 or force_split) and not cfg.host_staged
         self.side = torch.cuda.Stream()
         self.fork_ev, self.join_ev = torch.cuda.Event(), torch.cuda.Event()
+        self.separate_calls = separate_calls
+        # batches far larger than L2: one ep_layout_dispatch call with the side stream (C4: 289.5 against 291.2 us
+        # per step with separate calls); at C3 the early-resident dispatch CTAs delay the pair half (59.8 against 56.7 us)
+        self.one_call_split = self.split_layout and not separate_calls and not is_small(cfg)
         # decode-size batches: layout and dispatch in one launch (ep_layout_dispatch)
         self.fused = (not separate_calls) and T <= 1024 and not cfg.host_staged
         self.one_call = one_call and not self.fused and not cfg.host_staged
         if self.one_call:
-            self.split_layout = False
+            self.split_layout = self.one_call_split = False
 
     def step(self, ev=None):
         """layout -> dispatch -> combine. Dispatch needs only the receive-row half of the layout, so for big
@@ -298,6 +303,11 @@ class Workload:
         main = torch.cuda.current_stream()
         if ev:
             ev["t0"].record()
+        if self.one_call_split and ev is None:
+            # one call: receive-row half, dispatch launched behind it, pair half on the side stream, joined at the end
+            ep.ep_layout_dispatch(self.idx, self.x, self.recv, E, R, lay, self.ws_both, stream_pairs=self.side)
+            ep.ep_combine(self.out, lay.pair_slot, self.w, self.y, E, R, status=lay.status)
+            return
         if self.fused or self.one_call:
             ep.ep_layout_dispatch(self.idx, self.x, self.recv, E, R, lay, self.ws)    # small batches: one launch for both
         elif not self.split_layout:
@@ -547,7 +557,9 @@ def measure(ep, wl, steps, warmup, rep, no_graph=False, sample_clocks=True):
             "n_recv": n_recv, "n_pairs": n_pairs, "alg": alg, "launch": launch_note,
             "layout": "ep_layout_dispatch (layout and dispatch in one launch)" if wl.fused else
             "one ep_layout call" if not wl.split_layout else
-            "ep_layout_ranks before dispatch, ep_layout_pairs on a side stream beside dispatch",
+            ("ep_layout_dispatch with a second stream (receive-row half, dispatch launched behind it, pair half on the "
+             "side stream); the per-kernel pass issues the same work as separate calls" if wl.one_call_split else
+             "ep_layout_ranks before dispatch, ep_layout_pairs on a side stream beside dispatch"),
             "clocks": clocks.summary() if clocks else None}
 
 
@@ -836,7 +848,7 @@ def main():
     ap.add_argument("--serial-layout", action="store_true",
                     help="one ep_layout call instead of the receive-row half before dispatch and the pair half beside it")
     ap.add_argument("--separate-calls", action="store_true",
-                    help="small batches: ep_layout and ep_dispatch as two calls instead of ep_layout_dispatch")
+                    help="ep_layout (or its halves) and ep_dispatch as separate calls instead of ep_layout_dispatch")
     ap.add_argument("--force-split", action="store_true", help="split layout (pair half on a side stream) also for small batches")
     ap.add_argument("--one-call", action="store_true",
                     help="big batches: ep_layout_dispatch (whole layout, dispatch launched behind it with programmatic "

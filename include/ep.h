@@ -178,13 +178,22 @@ int ep_dispatch(const ep_shape_t *shape, const void *x, const int32_t *recv_slot
  * word (EP_STATUS_BAD_INDEX, EP_STATUS_CAPACITY when N_recv exceeds
  * recv_capacity_rows). Batches of up to 1024 tokens whose routing table fits in
  * shared memory take one launch in which every CTA derives the layout for itself
- * and moves its own tokens' rows; larger batches run the two calls one after the
- * other. Arguments as for ep_layout and ep_dispatch; the workspace is only used
- * by the larger batches.
+ * and moves its own tokens' rows. Larger batches run the layout kernels and
+ * then the dispatch kernel, launched so that its CTAs load their rows of x while
+ * the layout still runs (x and topk_idx are inputs of this call: they must be
+ * complete on `stream` before it). stream_pairs (may be NULL) is a second
+ * stream for those larger batches: the pair half of the layout, which dispatch
+ * does not need, then runs there beside dispatch; the call orders it behind what
+ * is queued on `stream` and makes `stream` wait for it at the end, so that on
+ * return everything is ordered on `stream` as if it had run there. With
+ * stream_pairs the workspace must hold 2 * ep_layout_workspace_bytes() + 256
+ * bytes (EP_ERR_CAPACITY otherwise); batches of up to 1024 tokens use neither.
+ * The two ordering events come from the library's pool (see the host-staged
+ * conventions below).
  */
 int ep_layout_dispatch(const ep_shape_t *shape, const int32_t *topk_idx, const void *x, const ep_layout_t *out,
                        void *workspace, size_t workspace_bytes, void *recv, int64_t recv_capacity_rows,
-                       void *stream);
+                       void *stream, void *stream_pairs);
 
 /*
  * Combine (Section 1; Section 4.3: the contributions that arrive for a token are

@@ -21,6 +21,7 @@
 //      expert_offsets[e] + (pairs of e before t0);
 //   5. all warps copy the own rows to their distinct destinations.
 #include <atomic>
+#include <mutex>
 
 #include "ep_common.cuh"
 #include "ep_layout_common.cuh"
@@ -278,7 +279,7 @@ __global__ void __launch_bounds__(kFusedThreads) layout_dispatch_small_kernel(Fu
 
 extern "C" int ep_layout_dispatch(const ep_shape_t *shape, const int32_t *topk_idx, const void *x,
                                   const ep_layout_t *out, void *workspace, size_t workspace_bytes, void *recv,
-                                  int64_t recv_capacity_rows, void *stream_)
+                                  int64_t recv_capacity_rows, void *stream_, void *stream_pairs_)
 {
     using namespace ep;
     int rc = check_shape(shape, true);
@@ -288,13 +289,36 @@ extern "C" int ep_layout_dispatch(const ep_shape_t *shape, const int32_t *topk_i
         // larger batches: the layout, then the dispatch kernel launched with programmatic stream serialisation,
         // so that its CTAs load their rows of x (an input of this call, complete before the layout starts)
         // while the layout still runs, and wait for the slots on the device
-        rc = ep_layout(shape, topk_idx, out, workspace, workspace_bytes, stream_);
-        if (rc != EP_OK) return rc;
+        cudaStream_t stream = static_cast<cudaStream_t>(stream_), side = static_cast<cudaStream_t>(stream_pairs_);
+        const bool split = stream_pairs_ != nullptr && shape->num_tokens > 0;
+        cudaEvent_t *ev = nullptr;
+        std::unique_lock<std::mutex> hold;
+        if (split) {
+            // dispatch needs the receive-row half only: the pair half runs on the second stream beside it
+            const size_t need = ep_layout_workspace_bytes(shape);
+            const size_t half = (need + 255) & ~size_t(255);
+            if (!workspace) return EP_ERR_NULL;
+            if (workspace_bytes < half + need) return EP_ERR_CAPACITY;
+            rc = order_events(&ev, 2, hold);
+            if (rc != EP_OK) return rc;
+            EP_CUDA_TRY(cudaEventRecord(ev[0], stream));                    // everything queued so far, x and topk_idx included
+            EP_CUDA_TRY(cudaStreamWaitEvent(side, ev[0], 0));
+            rc = ep_layout_ranks(shape, topk_idx, out, workspace, need, stream_);
+            if (rc != EP_OK) return rc;
+            rc = ep_layout_pairs(shape, topk_idx, out, static_cast<char *>(workspace) + half, need, stream_pairs_);
+            if (rc != EP_OK) return rc;
+            EP_CUDA_TRY(cudaEventRecord(ev[1], side));
+        } else {
+            rc = ep_layout(shape, topk_idx, out, workspace, workspace_bytes, stream_);
+            if (rc != EP_OK) return rc;
+        }
         if (shape->num_tokens == 0) return EP_OK;
         if (!x || !recv) return EP_ERR_NULL;
         if (!aligned16(x) || !aligned16(recv) || recv_capacity_rows < 0) return EP_ERR_INVALID_ARG;
-        return launch_dispatch(*shape, x, out->recv_slot, recv, recv_capacity_rows, out->status,
-                               static_cast<cudaStream_t>(stream_), true);
+        rc = launch_dispatch(*shape, x, out->recv_slot, recv, recv_capacity_rows, out->status, stream, true);
+        if (rc != EP_OK) return rc;
+        if (split) EP_CUDA_TRY(cudaStreamWaitEvent(stream, ev[1], 0));      // the pair half is part of this call's result
+        return EP_OK;
     }
     if (!out || !topk_idx || !x || !recv) return EP_ERR_NULL;
     if (!out->expert_counts || !out->expert_offsets || !out->rank_rows || !out->rank_row_offsets ||

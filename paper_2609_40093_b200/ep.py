@@ -72,7 +72,7 @@ def lib() -> ctypes.CDLL:
         L.ep_layout_static.restype = i32
         L.ep_layout_static_scratch_bytes.restype = sz
         L.ep_dispatch.argtypes = [sp, vp, vp, vp, i64, vp, vp]
-        L.ep_layout_dispatch.argtypes = [sp, vp, vp, ctypes.POINTER(_Layout), vp, sz, vp, i64, vp]
+        L.ep_layout_dispatch.argtypes = [sp, vp, vp, ctypes.POINTER(_Layout), vp, sz, vp, i64, vp, vp]
         L.ep_layout_dispatch.restype = i32
         L.ep_combine.argtypes = [sp, vp, i64, vp, vp, vp, vp, vp]
         L.ep_group.argtypes = [sp, vp, i64, vp, vp, vp, i64, vp, vp]
@@ -217,13 +217,15 @@ def ep_layout_static_scratch_bytes() -> int:
 
 
 def ep_layout_dispatch(topk_idx: torch.Tensor, x: torch.Tensor, recv: torch.Tensor, E: int, R: int, out: Layout,
-                       workspace: torch.Tensor) -> Layout:
-    """`ep_layout` followed by `ep_dispatch`, one launch for batches of up to 1024 tokens."""
+                       workspace: torch.Tensor, stream_pairs=None) -> Layout:
+    """`ep_layout` followed by `ep_dispatch`: one launch for batches of up to 1024 tokens; for larger ones
+    dispatch is launched behind the layout, whose pair half runs on `stream_pairs` (a torch stream) if given."""
     _want(topk_idx, torch.int32, "topk_idx"), _want(x, torch.bfloat16, "x"), _want(recv, torch.bfloat16, "recv")
     T, K = topk_idx.shape
     st = out.as_struct()
     _check(lib().ep_layout_dispatch(ctypes.byref(_shape(T, K, x.shape[1], E, R)), _ptr(topk_idx), _ptr(x), ctypes.byref(st),
-                                    _ptr(workspace), workspace.numel(), _ptr(recv), recv.shape[0], _stream()),
+                                    _ptr(workspace), workspace.numel(), _ptr(recv), recv.shape[0], _stream(),
+                                    ctypes.c_void_p(stream_pairs.cuda_stream) if stream_pairs is not None else None),
            "ep_layout_dispatch")
     return out
 

@@ -483,3 +483,38 @@ def test_small_step_with_the_fused_call_replays_from_a_cuda_graph():
         want = oracle.combine_f32(oracle.dispatch(d["x"], ref.recv_slot, ref.n_recv), ref.recv_slot, d["topk_weights"])
         np.testing.assert_array_equal(host_bits(y), want)
         assert ep.ep_status(lay.status) == 0
+
+
+@pytest.mark.parametrize("name", ["C3", "C4"])
+def test_layout_and_dispatch_in_one_call_with_a_second_stream(name):
+    """Prefill-size batches: the receive-row half and the dispatch kernel (launched behind it with programmatic
+    stream serialisation) on the main stream, the pair half on a second stream, everything ordered on the main
+    stream when the call returns. Three calls back to back on changing inputs, then the oracle's answers."""
+    cfg = inputs.CONFIGS[name]
+    T, K, H, E, R = cfg.T, cfg.K, cfg.H, cfg.E, cfg.R
+    one = max(16, ep.ep_layout_workspace_bytes(T, K, E, R))
+    ws = torch.empty(2 * one + 256, dtype=torch.uint8, device="cuda")
+    side = torch.cuda.Stream()
+    lay = ep.alloc_layout(T, K, E, R, fill=-7)
+    recv = torch.zeros(T * min(K, R), H, dtype=torch.bfloat16, device="cuda")
+    y = torch.zeros(T, H, dtype=torch.bfloat16, device="cuda")
+    idx_d = torch.zeros(T, K, dtype=torch.int32, device="cuda")
+    x_d = torch.zeros(T, H, dtype=torch.bfloat16, device="cuda")
+    for seed in (0, 1, 2):
+        d = inputs.make_inputs(cfg, seed)
+        idx = d["topk_idx"].copy()
+        idx[seed, 0] = -1
+        idx_d.copy_(torch.from_numpy(idx))
+        x_d.copy_(dev_bf16(d["x"]))
+        ep.ep_layout_dispatch(idx_d, x_d, recv, E, R, lay, ws, stream_pairs=side)
+        ep.ep_combine(recv, lay.recv_slot, torch.from_numpy(d["topk_weights"]).cuda(), y, E, R, status=lay.status)
+    torch.cuda.synchronize()
+    ref = oracle.layout(idx, E, R)
+    assert_layout_equal(lay, ref)
+    assert ep.ep_status(lay.status) == 0
+    want = oracle.dispatch(d["x"], ref.recv_slot, ref.n_recv)
+    np.testing.assert_array_equal(host_bits(recv)[:ref.n_recv], want)
+    np.testing.assert_array_equal(host_bits(y), oracle.combine_f32(want, ref.recv_slot, d["topk_weights"]))
+    with pytest.raises(ep.EPError) as err:                    # a second stream needs room for both halves' scratch
+        ep.ep_layout_dispatch(idx_d, x_d, recv, E, R, lay, ws[:one], stream_pairs=side)
+    assert err.value.code == -3
