@@ -432,20 +432,195 @@ extern "C" size_t ep_layout_workspace_bytes(const ep_shape_t *shape)
 namespace ep {
 namespace {
 
+// ---------------------------------------------------------------- receive-row half, lean form
+// The receive-row half alone (what dispatch waits for) for batches past the cluster form, compile-time
+// K and R <= 32: one token per lane with its picks in registers (vector loads, no staging in shared
+// memory), the exchange read by the whole CTA at once (one L2 round trip), one warp doing the scan over ranks
+// and the warps' bases, a pick's row looked up by its rank. Same two-kernel exchange as the general form:
+// the first kernel writes cta_part[cta][0..R] (rank hits, bad ids), the second is launched with
+// programmatic stream serialisation and waits on the device before it reads them.
+constexpr int kLeanWarps = 8;                       // 256 tokens per CTA
+constexpr int kLeanMaxCtas = 128;
+
+template <int KT>
+__device__ __forceinline__ void load_picks(const int32_t *idx, int t, int32_t (&e)[KT])
+{
+    if (KT % 4 == 0) {
+        const int4 *p = reinterpret_cast<const int4 *>(idx + (size_t)t * KT);
+#pragma unroll
+        for (int i = 0; i < KT / 4; ++i) {
+            const int4 v = __ldg(p + i);
+            e[4 * i] = v.x; e[4 * i + 1] = v.y; e[4 * i + 2] = v.z; e[4 * i + 3] = v.w;
+        }
+    } else {
+        const int2 *p = reinterpret_cast<const int2 *>(idx + (size_t)t * KT);
+#pragma unroll
+        for (int i = 0; i < KT / 2; ++i) {
+            const int2 v = __ldg(p + i);
+            e[2 * i] = v.x; e[2 * i + 1] = v.y;
+        }
+    }
+}
+
+// picks -> ranks (or -1), rank bitmask, number of ids outside [-1, E)
+template <int KT>
+__device__ __forceinline__ unsigned picks_to_ranks(const LayoutArgs &a, const int32_t (&e)[KT], int (&rk)[KT], int *bad)
+{
+    unsigned mask = 0u;
+#pragma unroll
+    for (int k = 0; k < KT; ++k) {
+        rk[k] = -1;
+        if ((unsigned)e[k] < (unsigned)a.E) {
+            rk[k] = sdiv(e[k], a.mul_El);
+            mask |= 1u << rk[k];
+        } else if (e[k] != -1) {
+            ++*bad;
+        }
+    }
+    return mask;
+}
+
+template <int KT, int RT>
+__global__ void __launch_bounds__(kLeanWarps * 32) ranks_count_kernel(LayoutArgs a)
+{
+    pdl_trigger();                                   // the second kernel may start its own loads now
+    __shared__ int32_t cnt[RT + 1];
+    const int tid = threadIdx.x, lane = tid & 31;
+    const int t = blockIdx.x * (kLeanWarps * 32) + tid;
+    if (tid <= RT) cnt[tid] = 0;
+    int32_t e[KT];
+    int rk[KT], bad = 0;
+#pragma unroll
+    for (int k = 0; k < KT; ++k) e[k] = -1;
+    if (t < a.T) load_picks<KT>(a.idx, t, e);
+    const unsigned mask = picks_to_ranks<KT>(a, e, rk, &bad);
+    __syncthreads();
+    int mine = 0;
+#pragma unroll
+    for (int r = 0; r < RT; ++r) {
+        const int c = __popc(__ballot_sync(kFullMask, (mask >> r) & 1u));
+        if (lane == r) mine = c;
+    }
+    if (lane < RT && mine) atomicAdd(cnt + lane, mine);
+    if (bad) atomicAdd(cnt + RT, bad);
+    __syncthreads();
+    if (tid <= RT) a.cta_part[(size_t)blockIdx.x * (RT + 1) + tid] = cnt[tid];
+}
+
+template <int KT, int RT>
+__global__ void __launch_bounds__(kLeanWarps * 32) ranks_assign_kernel(LayoutArgs a)
+{
+    pdl_trigger();
+    __shared__ int32_t wcnt[kLeanWarps][RT];         // rank hits per warp
+    __shared__ int32_t base[kLeanWarps][RT];         // first receive row of each warp's tokens per rank
+    __shared__ unsigned bal_s[kLeanWarps][RT];       // which of a warp's 32 tokens hit rank r
+    __shared__ int32_t acc[2][RT + 1];               // per rank (and bad ids): hits in earlier CTAs, hits in all
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int t = blockIdx.x * (kLeanWarps * 32) + tid;
+    const unsigned lt = lanemask_lt();
+    int32_t e[KT];
+    int rk[KT], bad = 0;
+#pragma unroll
+    for (int k = 0; k < KT; ++k) e[k] = -1;
+    if (t < a.T) load_picks<KT>(a.idx, t, e);
+    const unsigned mask = picks_to_ranks<KT>(a, e, rk, &bad);
+    unsigned bal[RT];
+#pragma unroll
+    for (int r = 0; r < RT; ++r) {
+        bal[r] = __ballot_sync(kFullMask, (mask >> r) & 1u);
+        if (lane == r) {
+            wcnt[warp][r] = __popc(bal[r]);
+            bal_s[warp][r] = bal[r];
+        }
+    }
+    if (tid < 2 * (RT + 1)) (&acc[0][0])[tid] = 0;
+    __syncthreads();
+    pdl_wait();                                      // cta_part is complete and visible
+    // every CTA's counters, all loads in flight at once (one L2 round trip), summed in shared memory
+    for (int i = tid; i < a.n_ctas * (RT + 1); i += kLeanWarps * 32) {
+        const int c = i / (RT + 1), r = i - c * (RT + 1);
+        const int32_t v = __ldcg(a.cta_part + i);
+        if (v) {
+            atomicAdd(&acc[1][r], v);
+            if (c < (int)blockIdx.x) atomicAdd(&acc[0][r], v);
+        }
+    }
+    __syncthreads();
+    if (warp == 0) {
+        // lane r < RT: rank r; lane RT: ids outside [-1, E)
+        const int32_t before = lane <= RT ? acc[0][lane] : 0, total = lane <= RT ? acc[1][lane] : 0;
+        const int32_t hits = lane < RT ? total : 0;
+        int32_t incl = hits;                         // scan over ranks: rank_row_offsets
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const int32_t up = __shfl_up_sync(kFullMask, incl, off);
+            if (lane >= off) incl += up;
+        }
+        const int32_t offset = incl - hits;
+        if (blockIdx.x == 0) {
+            if (lane < RT) {
+                a.out.rank_rows[lane] = total;
+                a.out.rank_row_offsets[lane] = offset;
+                a.out.src_row_offsets[lane * (RT + 1) + RT] = incl;
+            }
+            if (lane == RT) {
+                a.out.rank_row_offsets[RT] = offset;  // = the sum over all ranks
+                *a.out.status = total ? EP_STATUS_BAD_INDEX : 0;
+            }
+        }
+        if (lane < RT) {
+            int32_t run = offset + before;
+#pragma unroll
+            for (int w = 0; w < kLeanWarps; ++w) {
+                base[w][lane] = run;
+                run += wcnt[w][lane];
+            }
+        }
+    }
+    __syncthreads();
+    if (t >= a.T) return;
+    int32_t rows[KT];                                // receive row of every pick: looked up by its rank
+#pragma unroll
+    for (int k = 0; k < KT; ++k) rows[k] = rk[k] >= 0 ? base[warp][rk[k]] + __popc(bal_s[warp][rk[k]] & lt) : -1;
+    if (KT % 4 == 0) {
+        int4 *dst = reinterpret_cast<int4 *>(a.out.recv_slot + (size_t)t * KT);
+#pragma unroll
+        for (int i = 0; i < KT / 4; ++i) dst[i] = make_int4(rows[4 * i], rows[4 * i + 1], rows[4 * i + 2], rows[4 * i + 3]);
+    } else {
+        int2 *dst = reinterpret_cast<int2 *>(a.out.recv_slot + (size_t)t * KT);
+#pragma unroll
+        for (int i = 0; i < KT / 2; ++i) dst[i] = make_int2(rows[2 * i], rows[2 * i + 1]);
+    }
+    const int s = fdiv(t, a.by_Tr);
+    const bool first_of_source = t == s * a.Tr;      // where source rank s's segment starts in every rank
+#pragma unroll
+    for (int r = 0; r < RT; ++r) {
+        const int32_t row = base[warp][r] + __popc(bal[r] & lt);
+        if ((mask >> r) & 1u) a.out.recv_token[row] = t;   // a rank's rows of these 32 tokens are consecutive
+        if (first_of_source) a.out.src_row_offsets[r * (RT + 1) + s] = row;
+    }
+}
+
 // The kernels are compiled for the common (top-k, ranks) pairs with both as compile-time constants (their
 // loops unroll: the receive-row half of T=8192, K=8, R=8 takes 7.7 us instead of 9.4) and once with both
 // read at run time.
 using LayoutKernel = void (*)(LayoutArgs);
 struct KernelPair {
     LayoutKernel count, assign;
+    LayoutKernel ranks_count, ranks_assign;          // the lean receive-row form, NULL for run-time K and R
 };
 template <int KT, int RT>
-constexpr KernelPair kernel_pair() { return KernelPair{layout_cta_count_kernel<KT, RT>, layout_assign_kernel<KT, RT>}; }
+constexpr KernelPair kernel_pair()
+{
+    return KernelPair{layout_cta_count_kernel<KT, RT>, layout_assign_kernel<KT, RT>, ranks_count_kernel<KT, RT>,
+                      ranks_assign_kernel<KT, RT>};
+}
+constexpr KernelPair generic_pair() { return KernelPair{layout_cta_count_kernel<0, 0>, layout_assign_kernel<0, 0>, nullptr, nullptr}; }
 
 constexpr int kTunedTopK[] = {2, 4, 6, 8};
 constexpr int kTunedRanks = 8;
 constexpr int kNumKernelPairs = 5;
-const KernelPair kKernelPairs[kNumKernelPairs] = {kernel_pair<0, 0>(), kernel_pair<2, kTunedRanks>(), kernel_pair<4, kTunedRanks>(),
+const KernelPair kKernelPairs[kNumKernelPairs] = {generic_pair(), kernel_pair<2, kTunedRanks>(), kernel_pair<4, kTunedRanks>(),
                                                   kernel_pair<6, kTunedRanks>(), kernel_pair<8, kTunedRanks>()};
 
 int pick_kernels(int K, int R)
@@ -536,6 +711,15 @@ int run_layout(const ep_shape_t *shape, const int32_t *topk_idx, const ep_layout
         attr_done[dev].store(true, std::memory_order_release);
     }
     const int which = pick_kernels(shape->top_k, R);
+    if (parts == kPartRanks && kKernelPairs[which].ranks_assign && plan.mode != kModeSingle &&
+        ceil_div(T, kLeanWarps * 32) <= kLeanMaxCtas && aligned16(topk_idx) && aligned16(out->recv_slot)) {
+        // the receive-row half alone: the lean two-kernel form (cta_part holds R+1 counters per CTA)
+        a.n_ctas = ceil_div(T, kLeanWarps * 32);
+        kKernelPairs[which].ranks_count<<<a.n_ctas, kLeanWarps * 32, 0, stream>>>(a);
+        EP_CUDA_TRY(launch_pdl(kKernelPairs[which].ranks_assign, dim3(a.n_ctas), dim3(kLeanWarps * 32), 0, stream, a));
+        EP_LAUNCH_CHECK(2);
+        return EP_OK;
+    }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(plan.n_ctas);
     cfg.blockDim = dim3(plan.warps * 32);

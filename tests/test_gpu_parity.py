@@ -518,3 +518,30 @@ def test_layout_and_dispatch_in_one_call_with_a_second_stream(name):
     with pytest.raises(ep.EPError) as err:                    # a second stream needs room for both halves' scratch
         ep.ep_layout_dispatch(idx_d, x_d, recv, E, R, lay, ws[:one], stream_pairs=side)
     assert err.value.code == -3
+
+
+@pytest.mark.parametrize("K", [2, 4, 6, 8])
+def test_receive_row_half_on_the_lean_kernels(K):
+    """ep_layout_ranks with R = 8 and K in {2, 4, 6, 8} past 1024 tokens takes kernels of its own (picks in
+    registers, vector loads and stores). Ragged batch ends, masked / repeated / out-of-range ids, a batch too
+    large for them (falls back), and a routing table that is not 16-byte aligned (falls back)."""
+    rng = np.random.default_rng(20 + K)
+    R, E = 8, 64
+    for T in (1032, 2048, 4096 + 8, 8192, 32768, 40000):
+        idx = rng.integers(0, E, size=(T, K)).astype(np.int32)
+        idx[rng.random((T, K)) < 0.1] = -1
+        idx[7, :] = idx[7, 0]
+        idx[T - 1, K - 1] = E + 2
+        ref = oracle.layout(idx, E, R)
+        ws = torch.empty(max(16, ep.ep_layout_workspace_bytes(T, K, E, R)), dtype=torch.uint8, device="cuda")
+        for shift in (0, 1):                               # shift 1: the table starts 4 bytes past a 16-byte boundary
+            store = torch.zeros(T * K + 4, dtype=torch.int32, device="cuda")
+            idx_d = store[shift:shift + T * K].view(T, K)
+            idx_d.copy_(torch.from_numpy(idx))
+            lay = ep.alloc_layout(T, K, E, R, fill=-7)
+            ep.ep_layout_ranks(idx_d, E, R, lay, ws)
+            for f in ["rank_rows", "rank_row_offsets", "src_row_offsets", "recv_slot"]:
+                np.testing.assert_array_equal(getattr(lay, f).cpu().numpy(), getattr(ref, f), err_msg=f"{f} T={T} shift={shift}")
+            np.testing.assert_array_equal(lay.recv_token.cpu().numpy()[:ref.n_recv], ref.recv_token)
+            assert ep.ep_status(lay.status) == ep.STATUS_BAD_INDEX
+            assert (lay.pair_slot.cpu().numpy() == -7).all()   # the pair half is not this call's business
