@@ -496,19 +496,21 @@ def measure(ep, wl, steps, warmup, rep, no_graph=False, sample_clocks=True):
     inside the timed region. Small workloads: every step after an L2 flush, timed by its own event pair
     recorded inside a CUDA graph (small_in_graph), or with direct launches (small_direct)."""
     cfg, lay = wl.cfg, wl.lay
-    for _ in range(warmup):
-        wl.step()
+    small = is_small(cfg)
+    dev_index = torch.cuda.current_device()
+    clocks = ClockSampler(dev_index) if sample_clocks else None      # NVML set-up before the warm-up, not after it
+    wl.step()
     torch.cuda.synchronize()
     assert ep.ep_status(lay.status) == 0
     n_recv, n_pairs = int(lay.rank_row_offsets[-1]), int(lay.expert_offsets[-1])
     alg = algorithmic_bytes(cfg, n_recv, n_pairs)
-    small = is_small(cfg)
+    start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    for _ in range(warmup):                               # the W warm-up steps run right before the timed region
+        wl.step()
+    torch.cuda.synchronize()
     launches0 = ep.ep_launch_count()
-    dev_index = torch.cuda.current_device()
-    clocks = ClockSampler(dev_index) if sample_clocks else None
     if not small:
         # pass A, the timed region: K steps back to back, one event before and one after
-        start, stop = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         rep.barrier()
         if clocks:
             clocks.__enter__()
