@@ -432,15 +432,29 @@ extern "C" size_t ep_layout_workspace_bytes(const ep_shape_t *shape)
 namespace ep {
 namespace {
 
-// ---------------------------------------------------------------- receive-row half, lean form
-// The receive-row half alone (what dispatch waits for) for batches past the cluster form, compile-time
-// K and R <= 32: one token per lane with its picks in registers (vector loads, no staging in shared
-// memory), the exchange read by the whole CTA at once (one L2 round trip), one warp doing the scan over ranks
-// and the warps' bases, a pick's row looked up by its rank. Same two-kernel exchange as the general form:
-// the first kernel writes cta_part[cta][0..R] (rank hits, bad ids), the second is launched with
-// programmatic stream serialisation and waits on the device before it reads them.
+// ---------------------------------------------------------------- lean form
+// Batches past the one-CTA form with compile-time K and R <= 32 (and, for the pair half, E <= 1024): one token
+// per lane with its picks in registers (vector loads, no staging for the counting), the rank ballots in
+// registers, 256 tokens per CTA. Same two-kernel exchange as the general form: the first kernel writes
+// cta_part[cta] = [R rank-hit counters, bad ids | E expert counters], the second is launched with programmatic
+// stream serialisation and waits on the device before it reads them -- the rank counters with the whole CTA
+// at once (one L2 round trip, summed by shared-memory atomics: only sums are used), the expert counters one
+// expert per thread. One warp scans the ranks and sets the warps' receive-row bases while another scans the
+// experts; every pick's receive row is looked up by its rank; the slots leave as 16-byte stores. The pair
+// half replays each warp's 32*K pairs in (t,k) order from a staged copy, four 32-pair steps in flight, with
+// warp-private expert counters as in the general form.
+//   PAIRS == false: the receive-row half alone (what dispatch waits for), no dynamic shared memory;
+//   PAIRS == true : the pair half, or both halves (a.parts).
 constexpr int kLeanWarps = 8;                       // 256 tokens per CTA
 constexpr int kLeanMaxCtas = 128;
+constexpr int kLeanMaxExperts = 1024;
+constexpr int kLeanSteps = 4;
+
+inline size_t lean_smem_bytes(int E, int K)
+{
+    // ids_s[W][32*K] | rows_s[W][32*K] | whist[W][E] | tot[E+1] | before[E] | scan[32]
+    return sizeof(int32_t) * ((size_t)kLeanWarps * E + (E + 1) + E + 2 * (size_t)kLeanWarps * 32 * K + 32);
+}
 
 template <int KT>
 __device__ __forceinline__ void load_picks(const int32_t *idx, int t, int32_t (&e)[KT])
@@ -462,6 +476,20 @@ __device__ __forceinline__ void load_picks(const int32_t *idx, int t, int32_t (&
     }
 }
 
+// KT ints of one token to global or shared memory as 16- or 8-byte stores
+template <int KT>
+__device__ __forceinline__ void store_picks(int32_t *dst, const int32_t (&v)[KT])
+{
+    if (KT % 4 == 0) {
+#pragma unroll
+        for (int i = 0; i < KT / 4; ++i)
+            reinterpret_cast<int4 *>(dst)[i] = make_int4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
+    } else {
+#pragma unroll
+        for (int i = 0; i < KT / 2; ++i) reinterpret_cast<int2 *>(dst)[i] = make_int2(v[2 * i], v[2 * i + 1]);
+    }
+}
+
 // picks -> ranks (or -1), rank bitmask, number of ids outside [-1, E)
 template <int KT>
 __device__ __forceinline__ unsigned picks_to_ranks(const LayoutArgs &a, const int32_t (&e)[KT], int (&rk)[KT], int *bad)
@@ -480,14 +508,17 @@ __device__ __forceinline__ unsigned picks_to_ranks(const LayoutArgs &a, const in
     return mask;
 }
 
-template <int KT, int RT>
-__global__ void __launch_bounds__(kLeanWarps * 32) ranks_count_kernel(LayoutArgs a)
+template <int KT, int RT, bool PAIRS>
+__global__ void __launch_bounds__(kLeanWarps * 32) lean_count_kernel(LayoutArgs a)
 {
     pdl_trigger();                                   // the second kernel may start its own loads now
+    extern __shared__ int32_t dyn[];                 // PAIRS: this CTA's expert histogram [E]
     __shared__ int32_t cnt[RT + 1];
     const int tid = threadIdx.x, lane = tid & 31;
     const int t = blockIdx.x * (kLeanWarps * 32) + tid;
     if (tid <= RT) cnt[tid] = 0;
+    if (PAIRS)
+        for (int x = tid; x < a.E; x += kLeanWarps * 32) dyn[x] = 0;
     int32_t e[KT];
     int rk[KT], bad = 0;
 #pragma unroll
@@ -495,6 +526,11 @@ __global__ void __launch_bounds__(kLeanWarps * 32) ranks_count_kernel(LayoutArgs
     if (t < a.T) load_picks<KT>(a.idx, t, e);
     const unsigned mask = picks_to_ranks<KT>(a, e, rk, &bad);
     __syncthreads();
+    if (PAIRS) {
+#pragma unroll
+        for (int k = 0; k < KT; ++k)
+            if (rk[k] >= 0) atomicAdd(dyn + e[k], 1);
+    }
     int mine = 0;
 #pragma unroll
     for (int r = 0; r < RT; ++r) {
@@ -504,20 +540,36 @@ __global__ void __launch_bounds__(kLeanWarps * 32) ranks_count_kernel(LayoutArgs
     if (lane < RT && mine) atomicAdd(cnt + lane, mine);
     if (bad) atomicAdd(cnt + RT, bad);
     __syncthreads();
-    if (tid <= RT) a.cta_part[(size_t)blockIdx.x * (RT + 1) + tid] = cnt[tid];
+    int32_t *row = a.cta_part + (size_t)blockIdx.x * (RT + 1 + (PAIRS ? a.E : 0));
+    if (tid <= RT) row[tid] = cnt[tid];
+    if (PAIRS)
+        for (int x = tid; x < a.E; x += kLeanWarps * 32) row[RT + 1 + x] = dyn[x];
 }
 
-template <int KT, int RT>
-__global__ void __launch_bounds__(kLeanWarps * 32) ranks_assign_kernel(LayoutArgs a)
+template <int KT, int RT, bool PAIRS>
+__global__ void __launch_bounds__(kLeanWarps * 32) lean_assign_kernel(LayoutArgs a)
 {
     pdl_trigger();
+    extern __shared__ int32_t dyn[];
     __shared__ int32_t wcnt[kLeanWarps][RT];         // rank hits per warp
     __shared__ int32_t base[kLeanWarps][RT];         // first receive row of each warp's tokens per rank
     __shared__ unsigned bal_s[kLeanWarps][RT];       // which of a warp's 32 tokens hit rank r
     __shared__ int32_t acc[2][RT + 1];               // per rank (and bad ids): hits in earlier CTAs, hits in all
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int t = blockIdx.x * (kLeanWarps * 32) + tid;
+    const int tw = blockIdx.x * (kLeanWarps * 32) + warp * 32;   // this warp's first token
+    const int t = tw + lane;
     const unsigned lt = lanemask_lt();
+    const int E = a.E, stride = RT + 1 + (PAIRS ? E : 0);
+    const bool ranks = !PAIRS || (a.parts & kPartRanks);
+    // PAIRS: ids_s[W][32*KT] | rows_s[W][32*KT] (both written by 16-byte stores) | whist[W][E] | tot[E+1] | before[E] | scan[32]
+    int32_t *ids_s = dyn + warp * 32 * KT;
+    int32_t *rows_s = dyn + kLeanWarps * 32 * KT + warp * 32 * KT;
+    int32_t *hist = dyn + 2 * kLeanWarps * 32 * KT;  // [W][E]
+    int32_t *whist = hist + warp * E;                // this warp's expert counts, later next free pair slot
+    int32_t *tot = hist + kLeanWarps * E;
+    int32_t *before_e = tot + E + 1;
+    int32_t *sh = before_e + E;
+
     int32_t e[KT];
     int rk[KT], bad = 0;
 #pragma unroll
@@ -533,20 +585,42 @@ __global__ void __launch_bounds__(kLeanWarps * 32) ranks_assign_kernel(LayoutArg
             bal_s[warp][r] = bal[r];
         }
     }
+    if (PAIRS) {
+        for (int x = lane; x < E; x += 32) whist[x] = 0;
+        store_picks<KT>(ids_s + lane * KT, e);       // the warp's pairs in (t,k) order
+        __syncwarp();
+#pragma unroll
+        for (int k = 0; k < KT; ++k)
+            if (rk[k] >= 0) atomicAdd(whist + e[k], 1);
+    }
     if (tid < 2 * (RT + 1)) (&acc[0][0])[tid] = 0;
     __syncthreads();
     pdl_wait();                                      // cta_part is complete and visible
-    // every CTA's counters, all loads in flight at once (one L2 round trip), summed in shared memory
+    // rank counters of every CTA, all loads in flight at once, summed in shared memory
     for (int i = tid; i < a.n_ctas * (RT + 1); i += kLeanWarps * 32) {
         const int c = i / (RT + 1), r = i - c * (RT + 1);
-        const int32_t v = __ldcg(a.cta_part + i);
+        const int32_t v = __ldcg(a.cta_part + (size_t)c * stride + r);
         if (v) {
             atomicAdd(&acc[1][r], v);
             if (c < (int)blockIdx.x) atomicAdd(&acc[0][r], v);
         }
     }
+    if (PAIRS) {                                     // expert counters: one expert per thread, coalesced rows
+        for (int x = tid; x < E; x += kLeanWarps * 32) {
+            int32_t before = 0, total = 0;
+#pragma unroll 16
+            for (int c = 0; c < a.n_ctas; ++c) {
+                const int32_t v = __ldcg(a.cta_part + (size_t)c * stride + RT + 1 + x);
+                total += v;
+                if (c < (int)blockIdx.x) before += v;
+            }
+            tot[x] = total;
+            before_e[x] = before;
+            if (blockIdx.x == 0) a.out.expert_counts[x] = total;
+        }
+    }
     __syncthreads();
-    if (warp == 0) {
+    if (warp == (PAIRS ? 1 : 0)) {
         // lane r < RT: rank r; lane RT: ids outside [-1, E)
         const int32_t before = lane <= RT ? acc[0][lane] : 0, total = lane <= RT ? acc[1][lane] : 0;
         const int32_t hits = lane < RT ? total : 0;
@@ -557,7 +631,7 @@ __global__ void __launch_bounds__(kLeanWarps * 32) ranks_assign_kernel(LayoutArg
             if (lane >= off) incl += up;
         }
         const int32_t offset = incl - hits;
-        if (blockIdx.x == 0) {
+        if (blockIdx.x == 0 && ranks) {
             if (lane < RT) {
                 a.out.rank_rows[lane] = total;
                 a.out.rank_row_offsets[lane] = offset;
@@ -577,27 +651,79 @@ __global__ void __launch_bounds__(kLeanWarps * 32) ranks_assign_kernel(LayoutArg
             }
         }
     }
+    if (PAIRS) {
+        block_exclusive_scan_smem(tot, E, sh);       // tot[x] = expert offset, tot[E] = number of pairs
+        for (int x = tid; x < E; x += kLeanWarps * 32) {   // next free pair slot of expert x for every warp
+            int32_t run = tot[x] + before_e[x];
+#pragma unroll
+            for (int w = 0; w < kLeanWarps; ++w) {
+                const int32_t c = hist[w * E + x];
+                hist[w * E + x] = run;
+                run += c;
+            }
+        }
+        if (blockIdx.x == 0)
+            for (int x = tid; x <= E; x += kLeanWarps * 32) a.out.expert_offsets[x] = tot[x];
+    }
     __syncthreads();
-    if (t >= a.T) return;
+    const bool live = t < a.T;
     int32_t rows[KT];                                // receive row of every pick: looked up by its rank
 #pragma unroll
     for (int k = 0; k < KT; ++k) rows[k] = rk[k] >= 0 ? base[warp][rk[k]] + __popc(bal_s[warp][rk[k]] & lt) : -1;
-    if (KT % 4 == 0) {
-        int4 *dst = reinterpret_cast<int4 *>(a.out.recv_slot + (size_t)t * KT);
+    if (ranks && live) {
+        store_picks<KT>(a.out.recv_slot + (size_t)t * KT, rows);
+        const int s = fdiv(t, a.by_Tr);
+        const bool first_of_source = t == s * a.Tr;  // where source rank s's segment starts in every rank
 #pragma unroll
-        for (int i = 0; i < KT / 4; ++i) dst[i] = make_int4(rows[4 * i], rows[4 * i + 1], rows[4 * i + 2], rows[4 * i + 3]);
-    } else {
-        int2 *dst = reinterpret_cast<int2 *>(a.out.recv_slot + (size_t)t * KT);
-#pragma unroll
-        for (int i = 0; i < KT / 2; ++i) dst[i] = make_int2(rows[2 * i], rows[2 * i + 1]);
+        for (int r = 0; r < RT; ++r) {
+            const int32_t row = base[warp][r] + __popc(bal[r] & lt);
+            if ((mask >> r) & 1u) a.out.recv_token[row] = t;   // a rank's rows of these 32 tokens are consecutive
+            if (first_of_source) a.out.src_row_offsets[r * (RT + 1) + s] = row;
+        }
     }
-    const int s = fdiv(t, a.by_Tr);
-    const bool first_of_source = t == s * a.Tr;      // where source rank s's segment starts in every rank
+    if (!PAIRS) return;
+    store_picks<KT>(rows_s + lane * KT, rows);
+    __syncwarp();
+    // pair slots: the warp's 32*KT pairs in (t,k) order, kLeanSteps steps of 32 in flight
+    int32_t *pair_slot = a.out.pair_slot + (size_t)tw * KT;
+    for (int j0 = 0; j0 < KT; j0 += kLeanSteps) {
+        int ex[kLeanSteps], leader[kLeanSteps];
+        unsigned m[kLeanSteps];
+        int32_t first[kLeanSteps];
 #pragma unroll
-    for (int r = 0; r < RT; ++r) {
-        const int32_t row = base[warp][r] + __popc(bal[r] & lt);
-        if ((mask >> r) & 1u) a.out.recv_token[row] = t;   // a rank's rows of these 32 tokens are consecutive
-        if (first_of_source) a.out.src_row_offsets[r * (RT + 1) + s] = row;
+        for (int u = 0; u < kLeanSteps; ++u) {
+            const int i = 32 * (j0 + u) + lane;
+            ex[u] = j0 + u < KT ? ids_s[i] : -1;
+            if ((unsigned)ex[u] >= (unsigned)E) ex[u] = -1;
+        }
+#pragma unroll
+        for (int u = 0; u < kLeanSteps; ++u) {
+            m[u] = __match_any_sync(kFullMask, ex[u] >= 0 ? ex[u] : E + lane);
+            leader[u] = __ffs(m[u]) - 1;
+        }
+#pragma unroll
+        for (int u = 0; u < kLeanSteps; ++u) {
+            first[u] = 0;
+            if (ex[u] >= 0 && lane == leader[u]) first[u] = atomicAdd(whist + ex[u], __popc(m[u]));   // the group's slots at once
+            __syncwarp();                            // orders this step's counter update before the next step's
+        }
+#pragma unroll
+        for (int u = 0; u < kLeanSteps; ++u) {
+            const int i = 32 * (j0 + u) + lane;
+            const int tok = tw + i / KT;
+            first[u] = __shfl_sync(kFullMask, first[u], leader[u]);
+            if (j0 + u < KT && tok < a.T) {
+                if (ex[u] >= 0) {
+                    const int32_t p = first[u] + __popc(m[u] & lt);
+                    const int32_t row = rows_s[i];
+                    pair_slot[i] = p;
+                    a.out.pair_token[p] = tok;
+                    a.out.pair_row[p] = row;
+                } else {
+                    pair_slot[i] = -1;
+                }
+            }
+        }
     }
 }
 
@@ -607,15 +733,19 @@ __global__ void __launch_bounds__(kLeanWarps * 32) ranks_assign_kernel(LayoutArg
 using LayoutKernel = void (*)(LayoutArgs);
 struct KernelPair {
     LayoutKernel count, assign;
-    LayoutKernel ranks_count, ranks_assign;          // the lean receive-row form, NULL for run-time K and R
+    LayoutKernel ranks_count, ranks_assign;          // the lean form of the receive-row half, NULL for run-time K and R
+    LayoutKernel lean_count, lean_assign;            // the lean form of the pair half or of both halves
 };
 template <int KT, int RT>
 constexpr KernelPair kernel_pair()
 {
-    return KernelPair{layout_cta_count_kernel<KT, RT>, layout_assign_kernel<KT, RT>, ranks_count_kernel<KT, RT>,
-                      ranks_assign_kernel<KT, RT>};
+    return KernelPair{layout_cta_count_kernel<KT, RT>, layout_assign_kernel<KT, RT>, lean_count_kernel<KT, RT, false>,
+                      lean_assign_kernel<KT, RT, false>, lean_count_kernel<KT, RT, true>, lean_assign_kernel<KT, RT, true>};
 }
-constexpr KernelPair generic_pair() { return KernelPair{layout_cta_count_kernel<0, 0>, layout_assign_kernel<0, 0>, nullptr, nullptr}; }
+constexpr KernelPair generic_pair()
+{
+    return KernelPair{layout_cta_count_kernel<0, 0>, layout_assign_kernel<0, 0>, nullptr, nullptr, nullptr, nullptr};
+}
 
 constexpr int kTunedTopK[] = {2, 4, 6, 8};
 constexpr int kTunedRanks = 8;
@@ -707,16 +837,25 @@ int run_layout(const ep_shape_t *shape, const int32_t *topk_idx, const ep_layout
         for (int i = 0; i < kNumKernelPairs; ++i) {
             EP_CUDA_TRY(cudaFuncSetAttribute(kKernelPairs[i].count, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget));
             EP_CUDA_TRY(cudaFuncSetAttribute(kKernelPairs[i].assign, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget));
+            if (kKernelPairs[i].lean_assign)
+                EP_CUDA_TRY(cudaFuncSetAttribute(kKernelPairs[i].lean_assign, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                 (int)lean_smem_bytes(kLeanMaxExperts, kTunedTopK[i - 1])));
         }
         attr_done[dev].store(true, std::memory_order_release);
     }
     const int which = pick_kernels(shape->top_k, R);
-    if (parts == kPartRanks && kKernelPairs[which].ranks_assign && plan.mode != kModeSingle &&
-        ceil_div(T, kLeanWarps * 32) <= kLeanMaxCtas && aligned16(topk_idx) && aligned16(out->recv_slot)) {
-        // the receive-row half alone: the lean two-kernel form (cta_part holds R+1 counters per CTA)
+    if (kKernelPairs[which].ranks_assign && plan.mode != kModeSingle && ceil_div(T, kLeanWarps * 32) <= kLeanMaxCtas &&
+        aligned16(topk_idx) && (!ranks || aligned16(out->recv_slot)) && (!pairs || (aligned16(out->pair_slot) && E <= kLeanMaxExperts))) {
+        // the lean two-kernel form; cta_part holds R+1 (+E) counters per CTA, never more than the general form needs
         a.n_ctas = ceil_div(T, kLeanWarps * 32);
-        kKernelPairs[which].ranks_count<<<a.n_ctas, kLeanWarps * 32, 0, stream>>>(a);
-        EP_CUDA_TRY(launch_pdl(kKernelPairs[which].ranks_assign, dim3(a.n_ctas), dim3(kLeanWarps * 32), 0, stream, a));
+        const dim3 grid(a.n_ctas), block(kLeanWarps * 32);
+        if (!pairs) {
+            kKernelPairs[which].ranks_count<<<grid, block, 0, stream>>>(a);
+            EP_CUDA_TRY(launch_pdl(kKernelPairs[which].ranks_assign, grid, block, 0, stream, a));
+        } else {
+            kKernelPairs[which].lean_count<<<grid, block, sizeof(int32_t) * E, stream>>>(a);
+            EP_CUDA_TRY(launch_pdl(kKernelPairs[which].lean_assign, grid, block, lean_smem_bytes(E, shape->top_k), stream, a));
+        }
         EP_LAUNCH_CHECK(2);
         return EP_OK;
     }

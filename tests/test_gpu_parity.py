@@ -545,3 +545,34 @@ def test_receive_row_half_on_the_lean_kernels(K):
             np.testing.assert_array_equal(lay.recv_token.cpu().numpy()[:ref.n_recv], ref.recv_token)
             assert ep.ep_status(lay.status) == ep.STATUS_BAD_INDEX
             assert (lay.pair_slot.cpu().numpy() == -7).all()   # the pair half is not this call's business
+
+
+@pytest.mark.parametrize("K", [2, 4, 6, 8])
+def test_whole_layout_and_pair_half_on_the_lean_kernels(K):
+    """ep_layout and ep_layout_pairs with R = 8, K in {2, 4, 6, 8} and E <= 1024 past 1024 tokens take the lean
+    kernels too. Ragged batch ends, masked / repeated / out-of-range ids, 1024 experts, a batch and an expert
+    count too large for them (fall back), and a routing table that is not 16-byte aligned (falls back)."""
+    rng = np.random.default_rng(40 + K)
+    R = 8
+    for T, E in ((1032, 64), (2048, 8), (4096 + 8, 128), (8192, 256), (32768, 1024), (40000, 64), (2048, 2048)):
+        idx = rng.integers(0, E, size=(T, K)).astype(np.int32)
+        idx[rng.random((T, K)) < 0.1] = -1
+        idx[7, :] = idx[7, 0]
+        idx[T - 1, K - 1] = E + 2
+        ref = oracle.layout(idx, E, R)
+        ws = torch.empty(max(16, ep.ep_layout_workspace_bytes(T, K, E, R)), dtype=torch.uint8, device="cuda")
+        for shift in (0, 1):
+            store = torch.zeros(T * K + 4, dtype=torch.int32, device="cuda")
+            idx_d = store[shift:shift + T * K].view(T, K)
+            idx_d.copy_(torch.from_numpy(idx))
+            lay = ep.alloc_layout(T, K, E, R, fill=-7)
+            ep.ep_layout(idx_d, E, R, out=lay, workspace=ws)
+            assert_layout_equal(lay, ref)
+            assert ep.ep_status(lay.status) == ep.STATUS_BAD_INDEX
+            half = ep.alloc_layout(T, K, E, R, fill=-7)
+            ep.ep_layout_pairs(idx_d, E, R, half, ws)
+            for f in ["expert_counts", "expert_offsets", "pair_slot"]:
+                np.testing.assert_array_equal(getattr(half, f).cpu().numpy(), getattr(ref, f), err_msg=f"{f} T={T} E={E}")
+            np.testing.assert_array_equal(half.pair_row.cpu().numpy()[:ref.n_pairs], ref.pair_row)
+            np.testing.assert_array_equal(half.pair_token.cpu().numpy()[:ref.n_pairs], ref.pair_token)
+            assert (half.recv_slot.cpu().numpy() == -7).all() and int(half.status[0]) == -7   # not the pair half's business
