@@ -433,10 +433,10 @@ namespace ep {
 namespace {
 
 // ---------------------------------------------------------------- lean form
-// Batches past the one-CTA form with compile-time K and R <= 32 (and, for the pair half, E <= 1024): one token
+// Batches past the one-CTA form with compile-time K and at most RT ranks (and, for the pair half, E <= 1024): one token
 // per lane with its picks in registers (vector loads, no staging for the counting), the rank ballots in
-// registers, 256 tokens per CTA. Same two-kernel exchange as the general form: the first kernel writes
-// cta_part[cta] = [R rank-hit counters, bad ids | E expert counters], the second is launched with programmatic
+// registers, 256 tokens per CTA. Same two-kernel exchange as the general form, and the same scratch: the first
+// kernel writes cta_part[cta] = [R rank-hit counters | bad ids | E expert counters], the second is launched with programmatic
 // stream serialisation and waits on the device before it reads them -- the rank counters with the whole CTA
 // at once (one L2 round trip, summed by shared-memory atomics: only sums are used), the expert counters one
 // expert per thread. One warp scans the ranks and sets the warps' receive-row bases while another scans the
@@ -540,10 +540,13 @@ __global__ void __launch_bounds__(kLeanWarps * 32) lean_count_kernel(LayoutArgs 
     if (lane < RT && mine) atomicAdd(cnt + lane, mine);
     if (bad) atomicAdd(cnt + RT, bad);
     __syncthreads();
-    int32_t *row = a.cta_part + (size_t)blockIdx.x * (RT + 1 + (PAIRS ? a.E : 0));
-    if (tid <= RT) row[tid] = cnt[tid];
+    // one row per CTA, as wide as the general form's: [R rank-hit counters | bad ids | E expert counters]
+    const int R = a.num_ranks;
+    int32_t *row = a.cta_part + (size_t)blockIdx.x * (R + 1 + (PAIRS ? a.E : 0));
+    if (tid < R) row[tid] = cnt[tid];
+    if (tid == RT) row[R] = cnt[RT];
     if (PAIRS)
-        for (int x = tid; x < a.E; x += kLeanWarps * 32) row[RT + 1 + x] = dyn[x];
+        for (int x = tid; x < a.E; x += kLeanWarps * 32) row[R + 1 + x] = dyn[x];
 }
 
 template <int KT, int RT, bool PAIRS>
@@ -559,7 +562,7 @@ __global__ void __launch_bounds__(kLeanWarps * 32) lean_assign_kernel(LayoutArgs
     const int tw = blockIdx.x * (kLeanWarps * 32) + warp * 32;   // this warp's first token
     const int t = tw + lane;
     const unsigned lt = lanemask_lt();
-    const int E = a.E, stride = RT + 1 + (PAIRS ? E : 0);
+    const int E = a.E, R = a.num_ranks, stride = R + 1 + (PAIRS ? E : 0);    // R <= RT: ranks R..RT-1 are never hit
     const bool ranks = !PAIRS || (a.parts & kPartRanks);
     // PAIRS: ids_s[W][32*KT] | rows_s[W][32*KT] (both written by 16-byte stores) | whist[W][E] | tot[E+1] | before[E] | scan[32]
     int32_t *ids_s = dyn + warp * 32 * KT;
@@ -597,12 +600,13 @@ __global__ void __launch_bounds__(kLeanWarps * 32) lean_assign_kernel(LayoutArgs
     __syncthreads();
     pdl_wait();                                      // cta_part is complete and visible
     // rank counters of every CTA, all loads in flight at once, summed in shared memory
-    for (int i = tid; i < a.n_ctas * (RT + 1); i += kLeanWarps * 32) {
-        const int c = i / (RT + 1), r = i - c * (RT + 1);
+    for (int i = tid; i < a.n_ctas * (R + 1); i += kLeanWarps * 32) {
+        const int c = i / (R + 1), r = i - c * (R + 1);
         const int32_t v = __ldcg(a.cta_part + (size_t)c * stride + r);
+        const int slot = r < R ? r : RT;             // the counter behind the ranks holds the bad ids
         if (v) {
-            atomicAdd(&acc[1][r], v);
-            if (c < (int)blockIdx.x) atomicAdd(&acc[0][r], v);
+            atomicAdd(&acc[1][slot], v);
+            if (c < (int)blockIdx.x) atomicAdd(&acc[0][slot], v);
         }
     }
     if (PAIRS) {                                     // expert counters: one expert per thread, coalesced rows
@@ -610,7 +614,7 @@ __global__ void __launch_bounds__(kLeanWarps * 32) lean_assign_kernel(LayoutArgs
             int32_t before = 0, total = 0;
 #pragma unroll 16
             for (int c = 0; c < a.n_ctas; ++c) {
-                const int32_t v = __ldcg(a.cta_part + (size_t)c * stride + RT + 1 + x);
+                const int32_t v = __ldcg(a.cta_part + (size_t)c * stride + R + 1 + x);
                 total += v;
                 if (c < (int)blockIdx.x) before += v;
             }
@@ -632,13 +636,13 @@ __global__ void __launch_bounds__(kLeanWarps * 32) lean_assign_kernel(LayoutArgs
         }
         const int32_t offset = incl - hits;
         if (blockIdx.x == 0 && ranks) {
-            if (lane < RT) {
+            if (lane < R) {
                 a.out.rank_rows[lane] = total;
                 a.out.rank_row_offsets[lane] = offset;
-                a.out.src_row_offsets[lane * (RT + 1) + RT] = incl;
+                a.out.src_row_offsets[lane * (R + 1) + R] = incl;
             }
             if (lane == RT) {
-                a.out.rank_row_offsets[RT] = offset;  // = the sum over all ranks
+                a.out.rank_row_offsets[R] = offset;   // = the sum over all ranks
                 *a.out.status = total ? EP_STATUS_BAD_INDEX : 0;
             }
         }
@@ -678,7 +682,7 @@ __global__ void __launch_bounds__(kLeanWarps * 32) lean_assign_kernel(LayoutArgs
         for (int r = 0; r < RT; ++r) {
             const int32_t row = base[warp][r] + __popc(bal[r] & lt);
             if ((mask >> r) & 1u) a.out.recv_token[row] = t;   // a rank's rows of these 32 tokens are consecutive
-            if (first_of_source) a.out.src_row_offsets[r * (RT + 1) + s] = row;
+            if (first_of_source && r < R) a.out.src_row_offsets[r * (R + 1) + s] = row;
         }
     }
     if (!PAIRS) return;
@@ -753,9 +757,16 @@ constexpr int kNumKernelPairs = 5;
 const KernelPair kKernelPairs[kNumKernelPairs] = {generic_pair(), kernel_pair<2, kTunedRanks>(), kernel_pair<4, kTunedRanks>(),
                                                   kernel_pair<6, kTunedRanks>(), kernel_pair<8, kTunedRanks>()};
 
-int pick_kernels(int K, int R)
+int pick_kernels(int K, int R)               // the general kernels: exact (K, R)
 {
     if (R == kTunedRanks)
+        for (int i = 0; i < 4; ++i)
+            if (K == kTunedTopK[i]) return i + 1;
+    return 0;
+}
+int pick_lean(int K, int R)                  // the lean kernels: exact K, any R up to the compiled bound
+{
+    if (R <= kTunedRanks)
         for (int i = 0; i < 4; ++i)
             if (K == kTunedTopK[i]) return i + 1;
     return 0;
@@ -844,17 +855,19 @@ int run_layout(const ep_shape_t *shape, const int32_t *topk_idx, const ep_layout
         attr_done[dev].store(true, std::memory_order_release);
     }
     const int which = pick_kernels(shape->top_k, R);
-    if (kKernelPairs[which].ranks_assign && plan.mode != kModeSingle && ceil_div(T, kLeanWarps * 32) <= kLeanMaxCtas &&
-        aligned16(topk_idx) && (!ranks || aligned16(out->recv_slot)) && (!pairs || (aligned16(out->pair_slot) && E <= kLeanMaxExperts))) {
-        // the lean two-kernel form; cta_part holds R+1 (+E) counters per CTA, never more than the general form needs
+    const int lean = pick_lean(shape->top_k, R);
+    if (lean && plan.mode != kModeSingle && ceil_div(T, kLeanWarps * 32) <= kLeanMaxCtas &&
+        aligned16(topk_idx) && (!ranks || aligned16(out->recv_slot)) && (!pairs || (aligned16(out->pair_slot) && E <= kLeanMaxExperts)) &&
+        sizeof(int32_t) * (size_t)ceil_div(T, kLeanWarps * 32) * (R + 1 + (pairs ? E : 0)) <= workspace_bytes) {
+        // the lean two-kernel form; cta_part holds R+1 (+E) counters per CTA: what the general form's plan asked for
         a.n_ctas = ceil_div(T, kLeanWarps * 32);
         const dim3 grid(a.n_ctas), block(kLeanWarps * 32);
         if (!pairs) {
-            kKernelPairs[which].ranks_count<<<grid, block, 0, stream>>>(a);
-            EP_CUDA_TRY(launch_pdl(kKernelPairs[which].ranks_assign, grid, block, 0, stream, a));
+            kKernelPairs[lean].ranks_count<<<grid, block, 0, stream>>>(a);
+            EP_CUDA_TRY(launch_pdl(kKernelPairs[lean].ranks_assign, grid, block, 0, stream, a));
         } else {
-            kKernelPairs[which].lean_count<<<grid, block, sizeof(int32_t) * E, stream>>>(a);
-            EP_CUDA_TRY(launch_pdl(kKernelPairs[which].lean_assign, grid, block, lean_smem_bytes(E, shape->top_k), stream, a));
+            kKernelPairs[lean].lean_count<<<grid, block, sizeof(int32_t) * E, stream>>>(a);
+            EP_CUDA_TRY(launch_pdl(kKernelPairs[lean].lean_assign, grid, block, lean_smem_bytes(E, shape->top_k), stream, a));
         }
         EP_LAUNCH_CHECK(2);
         return EP_OK;

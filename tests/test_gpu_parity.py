@@ -553,8 +553,10 @@ def test_whole_layout_and_pair_half_on_the_lean_kernels(K):
     kernels too. Ragged batch ends, masked / repeated / out-of-range ids, 1024 experts, a batch and an expert
     count too large for them (fall back), and a routing table that is not 16-byte aligned (falls back)."""
     rng = np.random.default_rng(40 + K)
-    R = 8
-    for T, E in ((1032, 64), (2048, 8), (4096 + 8, 128), (8192, 256), (32768, 1024), (40000, 64), (2048, 2048)):
+    for T, E, R in ((1032, 64, 8), (2048, 8, 8), (4096 + 8, 128, 8), (8192, 256, 8), (32768, 1024, 8), (40000, 64, 8),
+                    (2048, 2048, 8), (3000, 30, 1), (3000, 30, 2), (4098, 63, 3), (2052, 12, 4), (2051 * 5 // 5 * 5, 35, 5),
+                    (4200, 49, 7), (2048, 48, 16)):
+        T -= T % R
         idx = rng.integers(0, E, size=(T, K)).astype(np.int32)
         idx[rng.random((T, K)) < 0.1] = -1
         idx[7, :] = idx[7, 0]
@@ -576,3 +578,35 @@ def test_whole_layout_and_pair_half_on_the_lean_kernels(K):
             np.testing.assert_array_equal(half.pair_row.cpu().numpy()[:ref.n_pairs], ref.pair_row)
             np.testing.assert_array_equal(half.pair_token.cpu().numpy()[:ref.n_pairs], ref.pair_token)
             assert (half.recv_slot.cpu().numpy() == -7).all() and int(half.status[0]) == -7   # not the pair half's business
+
+
+def test_layout_stays_inside_its_workspace():
+    """The scratch a layout call uses is exactly what ep_layout_workspace_bytes asks for: guard bytes on both
+    sides of a workspace of that size survive every form of the layout (one CTA, cluster, two kernels, lean
+    kernels with fewer ranks than they were compiled for, large expert counts)."""
+    rng = np.random.default_rng(77)
+    guard = 4096
+    for T, K, E, R in [(512, 2, 8, 8), (2048, 6, 128, 8), (1536, 3, 12, 4), (3000, 2, 30, 1), (4098, 2, 63, 3), (8192, 8, 256, 8),
+                       (4096, 4, 1024, 8), (4096, 8, 2048, 8), (40000, 2, 16, 8), (3200, 32, 4096, 64), (4200, 6, 49, 7)]:
+        T -= T % R
+        idx = rng.integers(-1, E, size=(T, K)).astype(np.int32)
+        ref = oracle.layout(idx, E, R)
+        need = max(16, ep.ep_layout_workspace_bytes(T, K, E, R))
+        need_pad = (need + 15) // 16 * 16
+        buf = torch.full((guard + need_pad + guard,), 0x5A, dtype=torch.uint8, device="cuda")
+        ws = buf[guard:guard + need]
+        idx_d = torch.from_numpy(idx).cuda()
+        for call in ("whole", "ranks", "pairs"):
+            lay = ep.alloc_layout(T, K, E, R, fill=-7)
+            if call == "whole":
+                ep.ep_layout(idx_d, E, R, out=lay, workspace=ws)
+                assert_layout_equal(lay, ref)
+            elif call == "ranks":
+                ep.ep_layout_ranks(idx_d, E, R, lay, ws)
+                np.testing.assert_array_equal(lay.recv_slot.cpu().numpy(), ref.recv_slot)
+            else:
+                ep.ep_layout_pairs(idx_d, E, R, lay, ws)
+                np.testing.assert_array_equal(lay.pair_slot.cpu().numpy(), ref.pair_slot)
+            torch.cuda.synchronize()
+            b = buf.cpu().numpy()
+            assert (b[:guard] == 0x5A).all() and (b[guard + need:] == 0x5A).all(), (T, K, E, R, call)
