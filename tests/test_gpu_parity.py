@@ -610,3 +610,51 @@ def test_layout_stays_inside_its_workspace():
             torch.cuda.synchronize()
             b = buf.cpu().numpy()
             assert (b[:guard] == 0x5A).all() and (b[guard + need:] == 0x5A).all(), (T, K, E, R, call)
+
+
+def _guarded_layout(T, K, E, R, guard=64, sentinel=-77):
+    """All output arrays of a layout carved from one buffer with `guard` sentinel words between them
+    (every array starts on a 16-byte boundary)."""
+    sizes = [E, E + 1, R, R + 1, R * (R + 1), T * K, T * K, T * min(K, R), T * K, T * K, 1]
+    starts, pos = [], guard
+    for n in sizes:
+        starts.append(pos)
+        pos += (max(1, n) + 3) // 4 * 4 + guard
+    buf = torch.full((pos,), sentinel, dtype=torch.int32, device="cuda")
+    shapes = [(E,), (E + 1,), (R,), (R + 1,), (R, R + 1), (T, K), (T, K), (T * min(K, R),), (T * K,), (T * K,), (1,)]
+    views = [buf[s:s + n].view(*shape) for s, n, shape in zip(starts, sizes, shapes)]
+    keep = torch.ones(pos, dtype=torch.bool)
+    for s, n in zip(starts, sizes):
+        keep[s:s + n] = False
+    return ep.Layout(*views), buf, keep.cuda(), sentinel
+
+
+def test_layout_writes_nothing_outside_its_output_arrays():
+    """Every form of the layout (one CTA, cluster, two general kernels, lean kernels, the one-launch
+    layout + dispatch) with its outputs carved from one guarded buffer: the words between the arrays and
+    the entries past N_recv / P keep their sentinel."""
+    rng = np.random.default_rng(78)
+    for T, K, E, R, H in [(96, 3, 12, 4, 64), (1000, 10, 512, 8, 64), (2048, 5, 40, 8, 8), (4096, 8, 128, 8, 8),
+                          (3000, 2, 30, 1, 8), (4098, 6, 63, 3, 8), (9000, 7, 64, 4, 8), (40000, 2, 16, 8, 8)]:
+        T -= T % R
+        idx = rng.integers(-1, E, size=(T, K)).astype(np.int32)
+        ref = oracle.layout(idx, E, R)
+        idx_d = torch.from_numpy(idx).cuda()
+        ws = torch.empty(max(16, ep.ep_layout_workspace_bytes(T, K, E, R)), dtype=torch.uint8, device="cuda")
+        calls = ["whole", "halves"] + (["one_launch"] if T <= 1024 else [])
+        for call in calls:
+            lay, buf, keep, sentinel = _guarded_layout(T, K, E, R)
+            if call == "whole":
+                ep.ep_layout(idx_d, E, R, out=lay, workspace=ws)
+            elif call == "halves":
+                ep.ep_layout_ranks(idx_d, E, R, lay, ws)
+                ep.ep_layout_pairs(idx_d, E, R, lay, ws)
+            else:
+                x_d = torch.zeros(T, H, dtype=torch.bfloat16, device="cuda")
+                recv = torch.zeros(max(1, ref.n_recv), H, dtype=torch.bfloat16, device="cuda")
+                ep.ep_layout_dispatch(idx_d, x_d, recv, E, R, lay, ws)
+            torch.cuda.synchronize()
+            assert_layout_equal(lay, ref)
+            assert bool((buf[keep] == sentinel).all()), (T, K, E, R, call)
+            assert bool((lay.recv_token[ref.n_recv:] == sentinel).all()) and bool((lay.pair_row[ref.n_pairs:] == sentinel).all())
+            assert bool((lay.pair_token[ref.n_pairs:] == sentinel).all())
