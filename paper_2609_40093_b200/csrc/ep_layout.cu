@@ -433,7 +433,7 @@ namespace ep {
 namespace {
 
 // ---------------------------------------------------------------- lean form
-// Batches past the one-CTA form with compile-time K and at most RT ranks (and, for the pair half, E <= 1024): one token
+// Batches past the one-CTA form with compile-time K and at most RT <= 32 ranks (and, for the pair half, E <= 1024): one token
 // per lane with its picks in registers (vector loads, no staging for the counting), the rank ballots in
 // registers, 256 tokens per CTA. Same two-kernel exchange as the general form, and the same scratch: the first
 // kernel writes cta_part[cta] = [R rank-hit counters | bad ids | E expert counters], the second is launched with programmatic
@@ -625,9 +625,8 @@ __global__ void __launch_bounds__(kLeanWarps * 32) lean_assign_kernel(LayoutArgs
     }
     __syncthreads();
     if (warp == (PAIRS ? 1 : 0)) {
-        // lane r < RT: rank r; lane RT: ids outside [-1, E)
-        const int32_t before = lane <= RT ? acc[0][lane] : 0, total = lane <= RT ? acc[1][lane] : 0;
-        const int32_t hits = lane < RT ? total : 0;
+        // lane r < R: rank r (RT <= 32 ranks fit one warp); acc[.][RT] holds the ids outside [-1, E)
+        const int32_t before = lane < R ? acc[0][lane] : 0, hits = lane < R ? acc[1][lane] : 0;
         int32_t incl = hits;                         // scan over ranks: rank_row_offsets
 #pragma unroll
         for (int off = 1; off < 32; off <<= 1) {
@@ -635,15 +634,16 @@ __global__ void __launch_bounds__(kLeanWarps * 32) lean_assign_kernel(LayoutArgs
             if (lane >= off) incl += up;
         }
         const int32_t offset = incl - hits;
+        const int32_t n_recv = __shfl_sync(kFullMask, incl, 31);
         if (blockIdx.x == 0 && ranks) {
             if (lane < R) {
-                a.out.rank_rows[lane] = total;
+                a.out.rank_rows[lane] = hits;
                 a.out.rank_row_offsets[lane] = offset;
                 a.out.src_row_offsets[lane * (R + 1) + R] = incl;
             }
-            if (lane == RT) {
-                a.out.rank_row_offsets[R] = offset;   // = the sum over all ranks
-                *a.out.status = total ? EP_STATUS_BAD_INDEX : 0;
+            if (lane == 0) {
+                a.out.rank_row_offsets[R] = n_recv;
+                *a.out.status = acc[1][RT] ? EP_STATUS_BAD_INDEX : 0;
             }
         }
         if (lane < RT) {
@@ -737,39 +737,47 @@ __global__ void __launch_bounds__(kLeanWarps * 32) lean_assign_kernel(LayoutArgs
 using LayoutKernel = void (*)(LayoutArgs);
 struct KernelPair {
     LayoutKernel count, assign;
-    LayoutKernel ranks_count, ranks_assign;          // the lean form of the receive-row half, NULL for run-time K and R
-    LayoutKernel lean_count, lean_assign;            // the lean form of the pair half or of both halves
 };
 template <int KT, int RT>
-constexpr KernelPair kernel_pair()
-{
-    return KernelPair{layout_cta_count_kernel<KT, RT>, layout_assign_kernel<KT, RT>, lean_count_kernel<KT, RT, false>,
-                      lean_assign_kernel<KT, RT, false>, lean_count_kernel<KT, RT, true>, lean_assign_kernel<KT, RT, true>};
-}
-constexpr KernelPair generic_pair()
-{
-    return KernelPair{layout_cta_count_kernel<0, 0>, layout_assign_kernel<0, 0>, nullptr, nullptr, nullptr, nullptr};
-}
+constexpr KernelPair kernel_pair() { return KernelPair{layout_cta_count_kernel<KT, RT>, layout_assign_kernel<KT, RT>}; }
 
 constexpr int kTunedTopK[] = {2, 4, 6, 8};
 constexpr int kTunedRanks = 8;
 constexpr int kNumKernelPairs = 5;
-const KernelPair kKernelPairs[kNumKernelPairs] = {generic_pair(), kernel_pair<2, kTunedRanks>(), kernel_pair<4, kTunedRanks>(),
+const KernelPair kKernelPairs[kNumKernelPairs] = {kernel_pair<0, 0>(), kernel_pair<2, kTunedRanks>(), kernel_pair<4, kTunedRanks>(),
                                                   kernel_pair<6, kTunedRanks>(), kernel_pair<8, kTunedRanks>()};
 
-int pick_kernels(int K, int R)               // the general kernels: exact (K, R)
+int pick_kernels(int K, int R)               // the general kernels: exact (K, R), else the run-time pair
 {
     if (R == kTunedRanks)
         for (int i = 0; i < 4; ++i)
             if (K == kTunedTopK[i]) return i + 1;
     return 0;
 }
-int pick_lean(int K, int R)                  // the lean kernels: exact K, any R up to the compiled bound
+
+// The lean kernels: exact K, any rank count up to the bound they were compiled for (8 or 32).
+struct LeanKernels {
+    LayoutKernel ranks_count, ranks_assign;          // the receive-row half alone
+    LayoutKernel count, assign;                      // the pair half, or both halves
+};
+template <int KT, int RT>
+constexpr LeanKernels lean_kernels()
 {
-    if (R <= kTunedRanks)
-        for (int i = 0; i < 4; ++i)
-            if (K == kTunedTopK[i]) return i + 1;
-    return 0;
+    return LeanKernels{lean_count_kernel<KT, RT, false>, lean_assign_kernel<KT, RT, false>, lean_count_kernel<KT, RT, true>,
+                       lean_assign_kernel<KT, RT, true>};
+}
+constexpr int kLeanRankBounds[] = {8, 32};
+const LeanKernels kLeanKernels[2][4] = {
+    {lean_kernels<2, 8>(), lean_kernels<4, 8>(), lean_kernels<6, 8>(), lean_kernels<8, 8>()},
+    {lean_kernels<2, 32>(), lean_kernels<4, 32>(), lean_kernels<6, 32>(), lean_kernels<8, 32>()}};
+
+const LeanKernels *pick_lean(int K, int R)
+{
+    for (int b = 0; b < 2; ++b)
+        if (R <= kLeanRankBounds[b])
+            for (int i = 0; i < 4; ++i)
+                if (K == kTunedTopK[i]) return &kLeanKernels[b][i];
+    return nullptr;
 }
 
 // Can `cfg` (one cluster = the whole grid) be resident on device `dev`? Asked once per device and
@@ -848,14 +856,15 @@ int run_layout(const ep_shape_t *shape, const int32_t *topk_idx, const ep_layout
         for (int i = 0; i < kNumKernelPairs; ++i) {
             EP_CUDA_TRY(cudaFuncSetAttribute(kKernelPairs[i].count, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget));
             EP_CUDA_TRY(cudaFuncSetAttribute(kKernelPairs[i].assign, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget));
-            if (kKernelPairs[i].lean_assign)
-                EP_CUDA_TRY(cudaFuncSetAttribute(kKernelPairs[i].lean_assign, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                 (int)lean_smem_bytes(kLeanMaxExperts, kTunedTopK[i - 1])));
         }
+        for (int b = 0; b < 2; ++b)
+            for (int i = 0; i < 4; ++i)
+                EP_CUDA_TRY(cudaFuncSetAttribute(kLeanKernels[b][i].assign, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                 (int)lean_smem_bytes(kLeanMaxExperts, kTunedTopK[i])));
         attr_done[dev].store(true, std::memory_order_release);
     }
     const int which = pick_kernels(shape->top_k, R);
-    const int lean = pick_lean(shape->top_k, R);
+    const LeanKernels *lean = pick_lean(shape->top_k, R);
     if (lean && plan.mode != kModeSingle && ceil_div(T, kLeanWarps * 32) <= kLeanMaxCtas &&
         aligned16(topk_idx) && (!ranks || aligned16(out->recv_slot)) && (!pairs || (aligned16(out->pair_slot) && E <= kLeanMaxExperts)) &&
         sizeof(int32_t) * (size_t)ceil_div(T, kLeanWarps * 32) * (R + 1 + (pairs ? E : 0)) <= workspace_bytes) {
@@ -863,11 +872,11 @@ int run_layout(const ep_shape_t *shape, const int32_t *topk_idx, const ep_layout
         a.n_ctas = ceil_div(T, kLeanWarps * 32);
         const dim3 grid(a.n_ctas), block(kLeanWarps * 32);
         if (!pairs) {
-            kKernelPairs[lean].ranks_count<<<grid, block, 0, stream>>>(a);
-            EP_CUDA_TRY(launch_pdl(kKernelPairs[lean].ranks_assign, grid, block, 0, stream, a));
+            lean->ranks_count<<<grid, block, 0, stream>>>(a);
+            EP_CUDA_TRY(launch_pdl(lean->ranks_assign, grid, block, 0, stream, a));
         } else {
-            kKernelPairs[lean].lean_count<<<grid, block, sizeof(int32_t) * E, stream>>>(a);
-            EP_CUDA_TRY(launch_pdl(kKernelPairs[lean].lean_assign, grid, block, lean_smem_bytes(E, shape->top_k), stream, a));
+            lean->count<<<grid, block, sizeof(int32_t) * E, stream>>>(a);
+            EP_CUDA_TRY(launch_pdl(lean->assign, grid, block, lean_smem_bytes(E, shape->top_k), stream, a));
         }
         EP_LAUNCH_CHECK(2);
         return EP_OK;

@@ -555,7 +555,7 @@ def test_whole_layout_and_pair_half_on_the_lean_kernels(K):
     rng = np.random.default_rng(40 + K)
     for T, E, R in ((1032, 64, 8), (2048, 8, 8), (4096 + 8, 128, 8), (8192, 256, 8), (32768, 1024, 8), (40000, 64, 8),
                     (2048, 2048, 8), (3000, 30, 1), (3000, 30, 2), (4098, 63, 3), (2052, 12, 4), (2051 * 5 // 5 * 5, 35, 5),
-                    (4200, 49, 7), (2048, 48, 16)):
+                    (4200, 49, 7), (2048, 48, 16), (4096 + 32, 1024, 32), (6144, 96, 24), (2048, 128, 64)):
         T -= T % R
         idx = rng.integers(0, E, size=(T, K)).astype(np.int32)
         idx[rng.random((T, K)) < 0.1] = -1
@@ -587,7 +587,8 @@ def test_layout_stays_inside_its_workspace():
     rng = np.random.default_rng(77)
     guard = 4096
     for T, K, E, R in [(512, 2, 8, 8), (2048, 6, 128, 8), (1536, 3, 12, 4), (3000, 2, 30, 1), (4098, 2, 63, 3), (8192, 8, 256, 8),
-                       (4096, 4, 1024, 8), (4096, 8, 2048, 8), (40000, 2, 16, 8), (3200, 32, 4096, 64), (4200, 6, 49, 7)]:
+                       (4096, 4, 1024, 8), (4096, 8, 2048, 8), (40000, 2, 16, 8), (3200, 32, 4096, 64), (4200, 6, 49, 7),
+                       (4096, 8, 256, 16), (8192, 4, 64, 32), (3000, 6, 60, 20)]:
         T -= T % R
         idx = rng.integers(-1, E, size=(T, K)).astype(np.int32)
         ref = oracle.layout(idx, E, R)
@@ -635,7 +636,8 @@ def test_layout_writes_nothing_outside_its_output_arrays():
     the entries past N_recv / P keep their sentinel."""
     rng = np.random.default_rng(78)
     for T, K, E, R, H in [(96, 3, 12, 4, 64), (1000, 10, 512, 8, 64), (2048, 5, 40, 8, 8), (4096, 8, 128, 8, 8),
-                          (3000, 2, 30, 1, 8), (4098, 6, 63, 3, 8), (9000, 7, 64, 4, 8), (40000, 2, 16, 8, 8)]:
+                          (3000, 2, 30, 1, 8), (4098, 6, 63, 3, 8), (9000, 7, 64, 4, 8), (40000, 2, 16, 8, 8),
+                          (4096, 8, 256, 16, 8), (8192, 4, 64, 32, 8)]:
         T -= T % R
         idx = rng.integers(-1, E, size=(T, K)).astype(np.int32)
         ref = oracle.layout(idx, E, R)
