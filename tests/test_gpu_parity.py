@@ -660,3 +660,70 @@ def test_layout_writes_nothing_outside_its_output_arrays():
             assert bool((buf[keep] == sentinel).all()), (T, K, E, R, call)
             assert bool((lay.recv_token[ref.n_recv:] == sentinel).all()) and bool((lay.pair_row[ref.n_pairs:] == sentinel).all())
             assert bool((lay.pair_token[ref.n_pairs:] == sentinel).all())
+
+
+def test_buffers_past_four_gib():
+    """Row buffers whose byte offsets do not fit 32 bits (receive space 4.9 GB, pair space 7.5 GB):
+    65536 tokens of 7168 elements, 8 of 256 experts on 8 ranks. The layout is compared in full; the
+    moved and combined rows on samples that include the last rows of every buffer. x holds random
+    bit patterns (NaNs included: dispatch and grouping move bits), `out` is a block of 2^15 seeded
+    rows repeated: 2^32 bytes is not a whole number of rows, so a truncated offset cannot land on
+    an equal row."""
+    T, H, E, K, R = 65536, 7168, 256, 8, 8
+    cfg = inputs.custom_config(T, H, E, K, R, routing="burst", config_id=61)
+    idx, w = inputs.make_topk_idx(cfg), inputs.make_topk_weights(cfg)
+    ref = oracle.layout(idx, E, R)
+    assert ref.n_recv * H * 2 > 1 << 32 and ref.n_pairs * H * 2 > 1 << 32
+    lay = _run_layout(idx, E, R)
+    assert_layout_equal(lay, ref)
+    rng = np.random.default_rng(61)
+    x = rng.integers(0, 1 << 16, size=(T, H), dtype=np.uint16)
+    x_d = dev_bf16(x)
+
+    def rows_of(buf, rows):
+        return host_bits(buf[torch.from_numpy(np.asarray(rows, dtype=np.int64)).cuda()])
+
+    def guards_ok(whole):
+        return bool((whole[:GUARD].view(torch.int16) == SENTINEL).all()) and \
+            bool((whole[-GUARD:].view(torch.int16) == SENTINEL).all())
+
+    # dispatch: the highest receive rows, rows around the 4 GiB mark, and a random sample
+    spare = 2
+    whole, recv = guarded(ref.n_recv + spare, H)
+    ep.ep_dispatch(x_d, lay.recv_slot, recv, E, R, status=lay.status)
+    mark = (1 << 32) // (2 * H)
+    rows = np.unique(np.concatenate([np.arange(ref.n_recv - 64, ref.n_recv), np.arange(mark - 32, mark + 32),
+                                     np.arange(64), rng.integers(0, ref.n_recv, 2048)]))
+    np.testing.assert_array_equal(rows_of(recv, rows), x[ref.recv_token[rows]])
+    assert (rows_of(recv, np.arange(ref.n_recv, ref.n_recv + spare)) == SENTINEL).all() and guards_ok(whole)
+    assert ep.ep_status(lay.status) == 0
+
+    # local grouping into the pair space, then (same buffer) independent expert outputs for combine
+    pwhole, pair_rows = guarded(ref.n_pairs, H)
+    ep.ep_group(recv, lay, pair_rows, E, R, status=lay.status)
+    pmark = mark
+    prows = np.unique(np.concatenate([np.arange(ref.n_pairs - 64, ref.n_pairs), np.arange(pmark - 32, pmark + 32),
+                                      np.arange(64), rng.integers(0, ref.n_pairs, 2048)]))
+    np.testing.assert_array_equal(rows_of(pair_rows, prows), x[ref.pair_token[prows]])
+    assert guards_ok(pwhole)
+    del recv, whole
+
+    block_rows = 1 << 15
+    block = inputs.make_out(cfg, block_rows, seed=2)
+    block_d = dev_bf16(block)
+    for first in range(0, ref.n_pairs, block_rows):
+        n = min(block_rows, ref.n_pairs - first)
+        pair_rows[first:first + n] = block_d[:n]
+    ywhole, y = guarded(T, H)
+    ep.ep_combine(pair_rows, lay.pair_slot, torch.from_numpy(w).cuda(), y, E, R, status=lay.status)
+    last_pairs = ref.pair_token[np.arange(ref.n_pairs - 256, ref.n_pairs)]      # tokens that read the last rows
+    toks = np.unique(np.concatenate([last_pairs, np.arange(32), np.arange(T - 32, T), rng.integers(0, T, 512)]))
+    used = np.unique(ref.pair_slot[toks])
+    used = used[used >= 0]
+    compact = np.searchsorted(used, ref.pair_slot[toks]).astype(np.int32)        # the sampled tokens' rows, renumbered
+    out_c = block[used % block_rows]
+    yb = rows_of(y, toks)
+    np.testing.assert_array_equal(yb, oracle.combine_f32(out_c, compact, w[toks]))
+    assert within_tolerance(yb, oracle.combine_f64(out_c, compact, w[toks])).all()
+    assert guards_ok(ywhole) and guards_ok(pwhole)
+    assert ep.ep_status(lay.status) == 0
