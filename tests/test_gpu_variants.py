@@ -84,3 +84,64 @@ def test_dense_allgather_and_reduce_scatter(T, H, E, K, R, routing, mask):
     np.testing.assert_array_equal(host_bits(y), want_y)
     assert guards_intact(dwhole) and guards_intact(ywhole) and ep.ep_status(status) == 0
     assert R * T >= ref.n_recv                                          # the dense form never moves fewer rows
+
+
+def test_variants_on_buffers_past_four_gib():
+    """65536 tokens of 7168 elements, 8 of 256 experts on 8 ranks: the dense buffers and the pair space hold
+    7.5 GB each, the partial rows 4.9 GB. Sampled tokens (those that use the last rows of every buffer among
+    them) against the oracle run on the sample as a batch of its own, its slots renumbered."""
+    T, H, E, K, R = 65536, 7168, 256, 8, 8
+    cfg = inputs.custom_config(T, H, E, K, R, routing="burst", config_id=91)
+    idx, w = inputs.make_topk_idx(cfg), inputs.make_topk_weights(cfg)
+    ref = oracle.layout(idx, E, R)
+    idx_d, w_d = torch.from_numpy(idx).cuda(), torch.from_numpy(w).cuda()
+    lay = ep.ep_layout(idx_d, E, R)
+    rng = np.random.default_rng(91)
+    block_rows = 1 << 15
+    block = inputs.make_out(cfg, block_rows, seed=3)
+    block_d = dev_bf16(block)
+
+    def rows_of(buf, rows):
+        return host_bits(buf[torch.from_numpy(np.asarray(rows, dtype=np.int64)).cuda()])
+
+    # dense all-gather: every rank's copy of every token
+    x = block[:, :]                                                    # 32768 seeded rows, repeated twice
+    x_d = block_d.repeat(T // block_rows, 1)
+    big = torch.empty(R * T, H, dtype=torch.bfloat16, device="cuda")
+    ep.ep_dense_allgather(x_d, big, K, E, R)
+    rows = np.unique(np.concatenate([np.arange(R * T - 64, R * T), np.arange(64), rng.integers(0, R * T, 4096)]))
+    np.testing.assert_array_equal(rows_of(big, rows), x[(rows % T) % block_rows])
+    del x_d
+
+    # expert outputs in the pair space: the seeded block repeated (2^32 bytes is not a whole number of rows)
+    assert ref.n_pairs == R * T
+    out = big
+    for first in range(0, ref.n_pairs, block_rows):
+        out[first:first + block_rows] = block_d
+    toks = np.unique(np.concatenate([ref.pair_token[-256:], ref.recv_token[-256:], np.arange(32), np.arange(T - 32, T),
+                                     rng.integers(0, T, 512)]))
+    toks = toks[:len(toks) - len(toks) % R]
+    used = np.unique(ref.pair_slot[toks])
+    pair_c = np.searchsorted(used, ref.pair_slot[toks]).astype(np.int32)
+    out_c = block[used % block_rows]
+    used_recv = np.unique(ref.recv_slot[toks])
+    recv_c = np.searchsorted(used_recv, ref.recv_slot[toks]).astype(np.int32)
+
+    status = torch.zeros(1, dtype=torch.int32, device="cuda")
+    partial = torch.empty(ref.n_recv, H, dtype=torch.bfloat16, device="cuda")
+    y = torch.empty(T, H, dtype=torch.bfloat16, device="cuda")
+    ep.ep_combine_partial(out, lay, w_d, partial, y, E, R, status=status)
+    want_partial, want_y = oracle.combine_partial(out_c, pair_c, recv_c, w[toks], len(used_recv))
+    np.testing.assert_array_equal(rows_of(partial, used_recv), want_partial)
+    np.testing.assert_array_equal(rows_of(y, toks), want_y)
+    del partial
+
+    dense = torch.empty(R * T, H, dtype=torch.bfloat16, device="cuda")
+    y.zero_()
+    ep.ep_dense_reduce_scatter(idx_d, out, lay.pair_slot, w_d, dense, y, E, R, status=status)
+    want_dense, want_y = oracle.dense_reduce_scatter(idx[toks], out_c, pair_c, w[toks], E, R)
+    n = len(toks)
+    dense_rows = (np.arange(R)[:, None] * T + toks[None, :]).ravel()   # dense[r*T + t] <-> sample's [r*n + i]
+    np.testing.assert_array_equal(rows_of(dense, dense_rows), want_dense)
+    np.testing.assert_array_equal(rows_of(y, toks), want_y)
+    assert ep.ep_status(status) == 0
