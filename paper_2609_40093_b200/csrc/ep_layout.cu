@@ -274,12 +274,7 @@ __global__ void __launch_bounds__(kMaxWarpsSingle * 32) layout_assign_kernel(Lay
                 if (c < (int)blockIdx.x) before += v;
             }
         } else if (a.mode == kModeGlobal) {
-#pragma unroll 16
-            for (int c = 0; c < a.n_ctas; ++c) {
-                const int32_t v = __ldcg(a.cta_part + (size_t)c * a.bins + b);
-                total += v;
-                if (c < (int)blockIdx.x) before += v;
-            }
+            column_sums<16>(a.cta_part + b, a.bins, a.n_ctas, blockIdx.x, a.T < 0, a.cta_part, &total, &before);
         } else {
             total = cta_tot[b];
         }
@@ -449,6 +444,7 @@ constexpr int kLeanWarps = 8;                       // 256 tokens per CTA
 constexpr int kLeanMaxCtas = 128;
 constexpr int kLeanMaxExperts = 1024;
 constexpr int kLeanSteps = 4;
+constexpr int kLeanExchangeBatch = 32;              // CTAs' expert counters a thread requests at once
 
 inline size_t lean_smem_bytes(int E, int K)
 {
@@ -611,13 +607,10 @@ __global__ void __launch_bounds__(kLeanWarps * 32) lean_assign_kernel(LayoutArgs
     }
     if (PAIRS) {                                     // expert counters: one expert per thread, coalesced rows
         for (int x = tid; x < E; x += kLeanWarps * 32) {
-            int32_t before = 0, total = 0;
-#pragma unroll 16
-            for (int c = 0; c < a.n_ctas; ++c) {
-                const int32_t v = __ldcg(a.cta_part + (size_t)c * stride + R + 1 + x);
-                total += v;
-                if (c < (int)blockIdx.x) before += v;
-            }
+            int32_t before, total;
+            const int32_t *col = a.cta_part + R + 1 + x;
+            if (a.n_ctas <= 16) column_sums<16>(col, stride, a.n_ctas, blockIdx.x, a.T < 0, a.cta_part, &total, &before);
+            else column_sums<kLeanExchangeBatch>(col, stride, a.n_ctas, blockIdx.x, a.T < 0, a.cta_part, &total, &before);
             tot[x] = total;
             before_e[x] = before;
             if (blockIdx.x == 0) a.out.expert_counts[x] = total;
