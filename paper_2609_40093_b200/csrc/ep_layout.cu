@@ -109,7 +109,7 @@ struct LayoutArgs {
     ep_layout_t out;
     int32_t *cta_part;  // [n_ctas][bins], global form only
     int T, top_k, E, num_ranks, Tr;
-    uint32_t mul_El, mul_K;
+    uint32_t mul_El, mul_K, mul_R1;   // multipliers of sdiv for E/R, K and R+1
     FastDiv by_Tr;
     int tile_tokens, n_tiles, bins, n_ctas, mode;
     int parts;   // kPartRanks | kPartPairs: which outputs this call writes
@@ -595,16 +595,19 @@ __global__ void __launch_bounds__(kLeanWarps * 32) lean_assign_kernel(LayoutArgs
     if (tid < 2 * (RT + 1)) (&acc[0][0])[tid] = 0;
     __syncthreads();
     pdl_wait();                                      // cta_part is complete and visible
-    // rank counters of every CTA, all loads in flight at once, summed in shared memory
-    for (int i = tid; i < a.n_ctas * (R + 1); i += kLeanWarps * 32) {
-        const int c = i / (R + 1), r = i - c * (R + 1);
-        const int32_t v = __ldcg(a.cta_part + (size_t)c * stride + r);
-        const int slot = r < R ? r : RT;             // the counter behind the ranks holds the bad ids
-        if (v) {
-            atomicAdd(&acc[1][slot], v);
-            if (c < (int)blockIdx.x) atomicAdd(&acc[0][slot], v);
-        }
+    // rank counters of every CTA: the first two per thread are requested here and summed (shared-memory atomics) behind
+    // the expert counters' batch, so that both exchanges share one L2 round trip
+    const int n_items = a.n_ctas * (R + 1);
+    int32_t rv[2];
+    int rc[2], rr[2];
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+        const int i = min(tid + u * kLeanWarps * 32, n_items - 1);
+        rc[u] = sdiv(i, a.mul_R1);
+        rr[u] = i - rc[u] * (R + 1);
+        rv[u] = __ldcg(a.cta_part + (size_t)rc[u] * stride + rr[u]);
     }
+    if (!PAIRS && a.T < 0 && tid == 0) *a.cta_part = (int32_t)clock64();   // never true: ends the basic block (see column_sums)
     if (PAIRS) {                                     // expert counters: one expert per thread, coalesced rows
         for (int x = tid; x < E; x += kLeanWarps * 32) {
             int32_t before, total;
@@ -616,8 +619,27 @@ __global__ void __launch_bounds__(kLeanWarps * 32) lean_assign_kernel(LayoutArgs
             if (blockIdx.x == 0) a.out.expert_counts[x] = total;
         }
     }
+#pragma unroll
+    for (int u = 0; u < 2; ++u) {
+        const int slot = rr[u] < R ? rr[u] : RT;     // the counter behind the ranks holds the bad ids
+        if (tid + u * kLeanWarps * 32 < n_items && rv[u]) {
+            atomicAdd(&acc[1][slot], rv[u]);
+            if (rc[u] < (int)blockIdx.x) atomicAdd(&acc[0][slot], rv[u]);
+        }
+    }
+    for (int i = tid + 2 * kLeanWarps * 32; i < n_items; i += kLeanWarps * 32) {    // more than 512 counters: the rest
+        const int c = sdiv(i, a.mul_R1), r = i - c * (R + 1);
+        const int32_t v = __ldcg(a.cta_part + (size_t)c * stride + r);
+        const int slot = r < R ? r : RT;
+        if (v) {
+            atomicAdd(&acc[1][slot], v);
+            if (c < (int)blockIdx.x) atomicAdd(&acc[0][slot], v);
+        }
+    }
     __syncthreads();
-    if (warp == (PAIRS ? 1 : 0)) {
+    // PAIRS: warp 1 scans the ranks and sets every warp's bases while warp 0 scans the experts. Otherwise every warp
+    // scans the ranks itself and sets its own bases: no serial section, no second block barrier.
+    if (!PAIRS || warp == 1) {
         // lane r < R: rank r (RT <= 32 ranks fit one warp); acc[.][RT] holds the ids outside [-1, E)
         const int32_t before = lane < R ? acc[0][lane] : 0, hits = lane < R ? acc[1][lane] : 0;
         int32_t incl = hits;                         // scan over ranks: rank_row_offsets
@@ -628,7 +650,7 @@ __global__ void __launch_bounds__(kLeanWarps * 32) lean_assign_kernel(LayoutArgs
         }
         const int32_t offset = incl - hits;
         const int32_t n_recv = __shfl_sync(kFullMask, incl, 31);
-        if (blockIdx.x == 0 && ranks) {
+        if (blockIdx.x == 0 && ranks && (PAIRS || warp == 0)) {
             if (lane < R) {
                 a.out.rank_rows[lane] = hits;
                 a.out.rank_row_offsets[lane] = offset;
@@ -641,10 +663,16 @@ __global__ void __launch_bounds__(kLeanWarps * 32) lean_assign_kernel(LayoutArgs
         }
         if (lane < RT) {
             int32_t run = offset + before;
+            if (PAIRS) {
 #pragma unroll
-            for (int w = 0; w < kLeanWarps; ++w) {
-                base[w][lane] = run;
-                run += wcnt[w][lane];
+                for (int w = 0; w < kLeanWarps; ++w) {
+                    base[w][lane] = run;
+                    run += wcnt[w][lane];
+                }
+            } else {
+#pragma unroll
+                for (int w = 0; w < kLeanWarps - 1; ++w) run += w < warp ? wcnt[w][lane] : 0;
+                base[warp][lane] = run;
             }
         }
     }
@@ -661,8 +689,10 @@ __global__ void __launch_bounds__(kLeanWarps * 32) lean_assign_kernel(LayoutArgs
         }
         if (blockIdx.x == 0)
             for (int x = tid; x <= E; x += kLeanWarps * 32) a.out.expert_offsets[x] = tot[x];
+        __syncthreads();
+    } else {
+        __syncwarp();
     }
-    __syncthreads();
     const bool live = t < a.T;
     int32_t rows[KT];                                // receive row of every pick: looked up by its rank
 #pragma unroll
@@ -835,7 +865,8 @@ int run_layout(const ep_shape_t *shape, const int32_t *topk_idx, const ep_layout
     a.out = *out;
     a.cta_part = static_cast<int32_t *>(workspace);
     a.T = T; a.top_k = shape->top_k; a.E = E; a.num_ranks = R; a.Tr = T / R;
-    a.mul_El = small_div_mul(E / R); a.mul_K = small_div_mul(shape->top_k); a.by_Tr = make_fastdiv(T / R);
+    a.mul_El = small_div_mul(E / R); a.mul_K = small_div_mul(shape->top_k); a.mul_R1 = small_div_mul(R + 1);
+    a.by_Tr = make_fastdiv(T / R);
     a.tile_tokens = plan.tile_tokens; a.n_tiles = plan.n_tiles; a.bins = plan.bins; a.n_ctas = plan.n_ctas;
     a.mode = plan.mode;
     a.parts = parts;
