@@ -594,46 +594,67 @@ __global__ void __launch_bounds__(kLeanWarps * 32) lean_assign_kernel(LayoutArgs
     }
     if (tid < 2 * (RT + 1)) (&acc[0][0])[tid] = 0;
     __syncthreads();
-    pdl_wait();                                      // cta_part is complete and visible
-    // rank counters of every CTA: the first two per thread are requested here and summed (shared-memory atomics) behind
-    // the expert counters' batch, so that both exchanges share one L2 round trip
-    const int n_items = a.n_ctas * (R + 1);
-    int32_t rv[2];
-    int rc[2], rr[2];
+    if (a.mode == kModeSingle) {
+        // one CTA holds the whole batch (at most 256 tokens): its own counters are the totals; no first kernel, no scratch
+        if (tid < RT) {
+            int32_t hits = 0;
 #pragma unroll
-    for (int u = 0; u < 2; ++u) {
-        const int i = min(tid + u * kLeanWarps * 32, n_items - 1);
-        rc[u] = sdiv(i, a.mul_R1);
-        rr[u] = i - rc[u] * (R + 1);
-        rv[u] = __ldcg(a.cta_part + (size_t)rc[u] * stride + rr[u]);
-    }
-    if (!PAIRS && a.T < 0 && tid == 0) *a.cta_part = (int32_t)clock64();   // never true: ends the basic block (see column_sums)
-    if (PAIRS) {                                     // expert counters: one expert per thread, coalesced rows
-        for (int x = tid; x < E; x += kLeanWarps * 32) {
-            int32_t before, total;
-            const int32_t *col = a.cta_part + R + 1 + x;
-            if (a.n_ctas <= 16) column_sums<16>(col, stride, a.n_ctas, blockIdx.x, a.T < 0, a.cta_part, &total, &before);
-            else column_sums<kLeanExchangeBatch>(col, stride, a.n_ctas, blockIdx.x, a.T < 0, a.cta_part, &total, &before);
-            tot[x] = total;
-            before_e[x] = before;
-            if (blockIdx.x == 0) a.out.expert_counts[x] = total;
+            for (int w = 0; w < kLeanWarps; ++w) hits += wcnt[w][tid];
+            acc[1][tid] = hits;
         }
-    }
+        if (bad) atomicAdd(&acc[1][RT], bad);
+        if (PAIRS) {
+            for (int x = tid; x < E; x += kLeanWarps * 32) {
+                int32_t total = 0;
 #pragma unroll
-    for (int u = 0; u < 2; ++u) {
-        const int slot = rr[u] < R ? rr[u] : RT;     // the counter behind the ranks holds the bad ids
-        if (tid + u * kLeanWarps * 32 < n_items && rv[u]) {
-            atomicAdd(&acc[1][slot], rv[u]);
-            if (rc[u] < (int)blockIdx.x) atomicAdd(&acc[0][slot], rv[u]);
+                for (int w = 0; w < kLeanWarps; ++w) total += hist[w * E + x];
+                tot[x] = total;
+                before_e[x] = 0;
+                a.out.expert_counts[x] = total;
+            }
         }
-    }
-    for (int i = tid + 2 * kLeanWarps * 32; i < n_items; i += kLeanWarps * 32) {    // more than 512 counters: the rest
-        const int c = sdiv(i, a.mul_R1), r = i - c * (R + 1);
-        const int32_t v = __ldcg(a.cta_part + (size_t)c * stride + r);
-        const int slot = r < R ? r : RT;
-        if (v) {
-            atomicAdd(&acc[1][slot], v);
-            if (c < (int)blockIdx.x) atomicAdd(&acc[0][slot], v);
+    } else {
+        pdl_wait();                                      // cta_part is complete and visible
+        // rank counters of every CTA: the first two per thread are requested here and summed (shared-memory atomics) behind
+        // the expert counters' batch, so that both exchanges share one L2 round trip
+        const int n_items = a.n_ctas * (R + 1);
+        int32_t rv[2];
+        int rc[2], rr[2];
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const int i = min(tid + u * kLeanWarps * 32, n_items - 1);
+            rc[u] = sdiv(i, a.mul_R1);
+            rr[u] = i - rc[u] * (R + 1);
+            rv[u] = __ldcg(a.cta_part + (size_t)rc[u] * stride + rr[u]);
+        }
+        if (!PAIRS && a.T < 0 && tid == 0) *a.cta_part = (int32_t)clock64();   // never true: ends the basic block (see column_sums)
+        if (PAIRS) {                                     // expert counters: one expert per thread, coalesced rows
+            for (int x = tid; x < E; x += kLeanWarps * 32) {
+                int32_t before, total;
+                const int32_t *col = a.cta_part + R + 1 + x;
+                if (a.n_ctas <= 16) column_sums<16>(col, stride, a.n_ctas, blockIdx.x, a.T < 0, a.cta_part, &total, &before);
+                else column_sums<kLeanExchangeBatch>(col, stride, a.n_ctas, blockIdx.x, a.T < 0, a.cta_part, &total, &before);
+                tot[x] = total;
+                before_e[x] = before;
+                if (blockIdx.x == 0) a.out.expert_counts[x] = total;
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 2; ++u) {
+            const int slot = rr[u] < R ? rr[u] : RT;     // the counter behind the ranks holds the bad ids
+            if (tid + u * kLeanWarps * 32 < n_items && rv[u]) {
+                atomicAdd(&acc[1][slot], rv[u]);
+                if (rc[u] < (int)blockIdx.x) atomicAdd(&acc[0][slot], rv[u]);
+            }
+        }
+        for (int i = tid + 2 * kLeanWarps * 32; i < n_items; i += kLeanWarps * 32) {    // more than 512 counters: the rest
+            const int c = sdiv(i, a.mul_R1), r = i - c * (R + 1);
+            const int32_t v = __ldcg(a.cta_part + (size_t)c * stride + r);
+            const int slot = r < R ? r : RT;
+            if (v) {
+                atomicAdd(&acc[1][slot], v);
+                if (c < (int)blockIdx.x) atomicAdd(&acc[0][slot], v);
+            }
         }
     }
     __syncthreads();
@@ -889,6 +910,16 @@ int run_layout(const ep_shape_t *shape, const int32_t *topk_idx, const ep_layout
     }
     const int which = pick_kernels(shape->top_k, R);
     const LeanKernels *lean = pick_lean(shape->top_k, R);
+    if (lean && T <= kLeanWarps * 32 && aligned16(topk_idx) && (!ranks || aligned16(out->recv_slot)) &&
+        (!pairs || (aligned16(out->pair_slot) && E <= kLeanMaxExperts))) {
+        // at most 256 tokens: the lean main kernel alone, one CTA
+        a.n_ctas = 1;
+        a.mode = kModeSingle;
+        if (!pairs) lean->ranks_assign<<<1, kLeanWarps * 32, 0, stream>>>(a);
+        else lean->assign<<<1, kLeanWarps * 32, lean_smem_bytes(E, shape->top_k), stream>>>(a);
+        EP_LAUNCH_CHECK(1);
+        return EP_OK;
+    }
     if (lean && plan.mode != kModeSingle && ceil_div(T, kLeanWarps * 32) <= kLeanMaxCtas &&
         aligned16(topk_idx) && (!ranks || aligned16(out->recv_slot)) && (!pairs || (aligned16(out->pair_slot) && E <= kLeanMaxExperts)) &&
         sizeof(int32_t) * (size_t)ceil_div(T, kLeanWarps * 32) * (R + 1 + (pairs ? E : 0)) <= workspace_bytes) {
