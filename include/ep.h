@@ -176,18 +176,21 @@ int ep_dispatch(const ep_shape_t *shape, const void *x, const int32_t *recv_slot
  * exactly what ep_layout followed by ep_dispatch (with status = out->status)
  * produces: every array of `out`, the dispatched rows in recv, and the status
  * word (EP_STATUS_BAD_INDEX, EP_STATUS_CAPACITY when N_recv exceeds
- * recv_capacity_rows). Batches of up to 1024 tokens whose routing table fits in
+ * recv_capacity_rows). The call runs the layout kernels and then the dispatch
+ * kernel, launched so that its CTAs load their rows of x while the layout still
+ * runs (x and topk_idx are inputs of this call: they must be complete on
+ * `stream` before it). Only batches of up to 1024 tokens that the layout's
+ * fastest kernels do not cover (an odd top-k or one above 8, more than 32
+ * ranks, tables that are not 16-byte aligned) and whose routing table fits in
  * shared memory take one launch in which every CTA derives the layout for itself
- * and moves its own tokens' rows. Larger batches run the layout kernels and
- * then the dispatch kernel, launched so that its CTAs load their rows of x while
- * the layout still runs (x and topk_idx are inputs of this call: they must be
- * complete on `stream` before it). stream_pairs (may be NULL) is a second
- * stream for those larger batches: the pair half of the layout, which dispatch
- * does not need, then runs there beside dispatch; the call orders it behind what
- * is queued on `stream` and makes `stream` wait for it at the end, so that on
- * return everything is ordered on `stream` as if it had run there. With
- * stream_pairs the workspace must hold 2 * ep_layout_workspace_bytes() + 256
- * bytes (EP_ERR_CAPACITY otherwise); batches of up to 1024 tokens use neither.
+ * and moves its own tokens' rows. stream_pairs (may be NULL) is a second
+ * stream for batches of more than 1024 tokens: the pair half of the layout,
+ * which dispatch does not need, then runs there beside dispatch; the call
+ * orders it behind what is queued on `stream` and makes `stream` wait for it at
+ * the end, so that on return everything is ordered on `stream` as if it had run
+ * there. With stream_pairs such a batch needs a workspace of
+ * 2 * ep_layout_workspace_bytes() + 256 bytes (EP_ERR_CAPACITY otherwise);
+ * batches of up to 1024 tokens ignore stream_pairs and need the plain size.
  * The two ordering events come from the library's pool (see the host-staged
  * conventions below).
  */

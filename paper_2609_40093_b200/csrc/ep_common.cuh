@@ -44,6 +44,10 @@ int order_events(cudaEvent_t **pool, int need, std::unique_lock<std::mutex> &hol
         EP_CUDA_TRY(cudaGetLastError());                    \
     } while (0)
 
+// Would ep_layout run this call on its lean kernels (ep_layout.cu)? Then the layout followed by a dependent dispatch
+// launch is faster than the one-launch form of ep_layout_dispatch at every batch size.
+bool layout_is_lean(const ep_shape_t &shape, const void *topk_idx, const ep_layout_t &out, size_t workspace_bytes);
+
 // Kernel launchers shared between the translation units (arguments already validated).
 int launch_dispatch(const ep_shape_t &s, const void *x, const int32_t *recv_slot, void *recv,
                     int64_t capacity_rows, int32_t *status, cudaStream_t stream, bool behind_layout = false);

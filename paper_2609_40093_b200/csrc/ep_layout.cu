@@ -56,6 +56,9 @@ constexpr int kSteps = 4;               // 32-pair steps of the replay whose lat
 
 enum { kModeSingle = 0, kModeCluster = 1, kModeGlobal = 2 };
 enum { kPartRanks = 1, kPartPairs = 2 };
+constexpr int kLeanTokensPerCta = 256;              // the lean kernels: 8 warps, one token per lane
+constexpr int kLeanMaxCtas = 128;
+constexpr int kLeanMaxExperts = 1024;
 
 struct LayoutPlan {
     int mode;
@@ -101,6 +104,12 @@ LayoutPlan make_plan(const ep_shape_t &s)
     // the cluster form needs no scratch, but falls back to the global form on a device that cannot
     // keep the whole cluster resident, so both ask for cta_part
     p.workspace_bytes = p.mode == kModeSingle ? 16 : sizeof(int32_t) * (size_t)p.n_ctas * p.bins;
+    // the lean kernel pair (256 tokens per CTA) takes over from 257 tokens on: one scratch row per CTA of its own
+    const int lean_ctas = ceil_div(T, kLeanTokensPerCta);
+    if (lean_ctas > 1 && lean_ctas <= kLeanMaxCtas) {
+        const size_t lean = sizeof(int32_t) * (size_t)lean_ctas * p.bins;
+        p.workspace_bytes = lean > p.workspace_bytes ? lean : p.workspace_bytes;
+    }
     return p;
 }
 
@@ -440,9 +449,7 @@ namespace {
 // warp-private expert counters as in the general form.
 //   PAIRS == false: the receive-row half alone (what dispatch waits for), no dynamic shared memory;
 //   PAIRS == true : the pair half, or both halves (a.parts).
-constexpr int kLeanWarps = 8;                       // 256 tokens per CTA
-constexpr int kLeanMaxCtas = 128;
-constexpr int kLeanMaxExperts = 1024;
+constexpr int kLeanWarps = kLeanTokensPerCta / 32;
 constexpr int kLeanSteps = 4;
 constexpr int kLeanExchangeBatch = 32;              // CTAs' expert counters a thread requests at once
 
@@ -824,6 +831,22 @@ const LeanKernels *pick_lean(int K, int R)
     return nullptr;
 }
 
+// Which form a call takes: the lean kernels need an even top-k of at most 8, at most 32 ranks, 16-byte aligned tables
+// and, for the pair half, at most 1024 experts; the kernel pair also one scratch row per CTA inside the workspace.
+enum { kGeneral = 0, kLeanSingle = 1, kLeanPair = 2 };
+int lean_form(const ep_shape_t &s, const void *topk_idx, const ep_layout_t &out, size_t workspace_bytes, int parts)
+{
+    const bool ranks = parts & kPartRanks, pairs = parts & kPartPairs;
+    const int T = s.num_tokens, E = s.num_experts, R = s.num_ranks;
+    if (!pick_lean(s.top_k, R) || !aligned16(topk_idx) || (ranks && !aligned16(out.recv_slot)) ||
+        (pairs && (!aligned16(out.pair_slot) || E > kLeanMaxExperts)))
+        return kGeneral;
+    if (T <= kLeanTokensPerCta) return kLeanSingle;
+    const int n_ctas = ceil_div(T, kLeanTokensPerCta);
+    if (n_ctas > kLeanMaxCtas || sizeof(int32_t) * (size_t)n_ctas * (R + 1 + (pairs ? E : 0)) > workspace_bytes) return kGeneral;
+    return kLeanPair;
+}
+
 // Can `cfg` (one cluster = the whole grid) be resident on device `dev`? Asked once per device and
 // (cluster size, CTA size, shared memory) and remembered; "no" sends the call to the global form.
 bool cluster_fits(int dev, int which, const cudaLaunchConfig_t &cfg)
@@ -910,8 +933,8 @@ int run_layout(const ep_shape_t *shape, const int32_t *topk_idx, const ep_layout
     }
     const int which = pick_kernels(shape->top_k, R);
     const LeanKernels *lean = pick_lean(shape->top_k, R);
-    if (lean && T <= kLeanWarps * 32 && aligned16(topk_idx) && (!ranks || aligned16(out->recv_slot)) &&
-        (!pairs || (aligned16(out->pair_slot) && E <= kLeanMaxExperts))) {
+    const int form = lean_form(*shape, topk_idx, *out, workspace_bytes, parts);
+    if (form == kLeanSingle) {
         // at most 256 tokens: the lean main kernel alone, one CTA
         a.n_ctas = 1;
         a.mode = kModeSingle;
@@ -920,11 +943,10 @@ int run_layout(const ep_shape_t *shape, const int32_t *topk_idx, const ep_layout
         EP_LAUNCH_CHECK(1);
         return EP_OK;
     }
-    if (lean && plan.mode != kModeSingle && ceil_div(T, kLeanWarps * 32) <= kLeanMaxCtas &&
-        aligned16(topk_idx) && (!ranks || aligned16(out->recv_slot)) && (!pairs || (aligned16(out->pair_slot) && E <= kLeanMaxExperts)) &&
-        sizeof(int32_t) * (size_t)ceil_div(T, kLeanWarps * 32) * (R + 1 + (pairs ? E : 0)) <= workspace_bytes) {
-        // the lean two-kernel form; cta_part holds R+1 (+E) counters per CTA: what the general form's plan asked for
+    if (form == kLeanPair) {
+        // cta_part holds R+1 (+E) counters per CTA
         a.n_ctas = ceil_div(T, kLeanWarps * 32);
+        a.mode = kModeGlobal;
         const dim3 grid(a.n_ctas), block(kLeanWarps * 32);
         if (!pairs) {
             lean->ranks_count<<<grid, block, 0, stream>>>(a);
@@ -971,6 +993,12 @@ int run_layout(const ep_shape_t *shape, const int32_t *topk_idx, const ep_layout
 }
 
 }  // namespace
+
+bool layout_is_lean(const ep_shape_t &shape, const void *topk_idx, const ep_layout_t &out, size_t workspace_bytes)
+{
+    return lean_form(shape, topk_idx, out, workspace_bytes, kPartRanks | kPartPairs) != kGeneral;
+}
+
 }  // namespace ep
 
 extern "C" int ep_layout(const ep_shape_t *shape, const int32_t *topk_idx, const ep_layout_t *out,

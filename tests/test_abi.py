@@ -121,9 +121,10 @@ def test_host_staged_calls_check_their_segment_tables_before_touching_a_gpu():
 
 
 def test_workspace_sizes_follow_the_launch_plan():
-    """One CTA up to 1024 tokens (no scratch), then one row of E+R+1 counters per CTA, at most 128 CTAs."""
+    """One CTA up to 256 tokens (no scratch), then one row of E+R+1 counters per CTA of 256 tokens, at most 128 CTAs."""
     ws = ep.ep_layout_workspace_bytes
-    assert ws(64, 2, 8, 2) == 16 and ws(1024, 8, 256, 8) == 16
+    assert ws(64, 2, 8, 2) == 16 and ws(256, 8, 256, 8) == 16
+    assert ws(264, 8, 256, 8) == 2 * (256 + 8 + 1) * 4 and ws(1024, 8, 256, 8) == 4 * (256 + 8 + 1) * 4
     assert ws(2048, 8, 256, 8) == 8 * (256 + 8 + 1) * 4       # 8 CTAs of 8 warps
     assert ws(8192, 8, 256, 8) == 32 * (256 + 8 + 1) * 4
     assert ws(65536, 8, 256, 8) == 128 * (256 + 8 + 1) * 4    # 128 CTAs, two 32-token groups per warp

@@ -399,7 +399,8 @@ def test_largest_config_in_full():
     _full_path_check(cfg, d["topk_idx"], d["topk_weights"], d["x"])
 
 
-FUSED = [  # T, H, E, K, R, routing: batches that take the one-launch layout + dispatch, and two that do not
+FUSED = [  # T, H, E, K, R, routing: ep_layout_dispatch on batches that take its one-launch form (odd K, K > 8 or
+           # R > 32, up to 1024 tokens), on batches the lean layout kernels take instead, and on larger ones
     (64, 256, 8, 2, 2, "uniform"),         # C1
     (256, 4096, 8, 2, 8, "uniform"),       # C2
     (1, 8, 1, 1, 1, "uniform"),
@@ -409,7 +410,9 @@ FUSED = [  # T, H, E, K, R, routing: batches that take the one-launch layout + d
     (40, 520, 16, 4, 1, "uniform"),        # R = 1, 40 tokens: a ragged last group
     (48, 72, 16, 3, 16, "uniform"),
     (1000, 136, 512, 10, 8, "zipf"),
-    (1024, 7168, 256, 8, 8, "burst"),      # the largest fused batch, long rows
+    (1024, 7168, 256, 8, 8, "burst"),      # four CTAs of the lean kernel pair, long rows
+    (1024, 7168, 256, 7, 8, "uniform"),    # the largest batch of the one-launch form, long rows
+    (520, 72, 64, 6, 8, "zipf"),           # three CTAs of the lean kernel pair, the last one ragged
     (320, 64, 4096, 4, 64, "uniform"),     # E and R at their maxima
     (64, 64, 64, 32, 32, "uniform"),       # K at its maximum
     (1023 - 1023 % 3, 40, 24, 5, 3, "zipf_identity"),
@@ -583,12 +586,13 @@ def test_whole_layout_and_pair_half_on_the_lean_kernels(K):
 def test_layout_stays_inside_its_workspace():
     """The scratch a layout call uses is exactly what ep_layout_workspace_bytes asks for: guard bytes on both
     sides of a workspace of that size survive every form of the layout (one CTA, cluster, two kernels, lean
-    kernels with fewer ranks than they were compiled for, large expert counts)."""
+    kernels alone and as a pair, with fewer ranks than they were compiled for, large expert counts)."""
     rng = np.random.default_rng(77)
     guard = 4096
     for T, K, E, R in [(512, 2, 8, 8), (2048, 6, 128, 8), (1536, 3, 12, 4), (3000, 2, 30, 1), (4098, 2, 63, 3), (8192, 8, 256, 8),
                        (4096, 4, 1024, 8), (4096, 8, 2048, 8), (40000, 2, 16, 8), (3200, 32, 4096, 64), (4200, 6, 49, 7),
-                       (4096, 8, 256, 16), (8192, 4, 64, 32), (3000, 6, 60, 20)]:
+                       (4096, 8, 256, 16), (8192, 4, 64, 32), (3000, 6, 60, 20),
+                       (200, 8, 256, 8), (256, 2, 8, 8), (264, 6, 1024, 8), (1000, 4, 64, 8), (1024, 8, 256, 32)]:
         T -= T % R
         idx = rng.integers(-1, E, size=(T, K)).astype(np.int32)
         ref = oracle.layout(idx, E, R)
@@ -637,7 +641,8 @@ def test_layout_writes_nothing_outside_its_output_arrays():
     rng = np.random.default_rng(78)
     for T, K, E, R, H in [(96, 3, 12, 4, 64), (1000, 10, 512, 8, 64), (2048, 5, 40, 8, 8), (4096, 8, 128, 8, 8),
                           (3000, 2, 30, 1, 8), (4098, 6, 63, 3, 8), (9000, 7, 64, 4, 8), (40000, 2, 16, 8, 8),
-                          (4096, 8, 256, 16, 8), (8192, 4, 64, 32, 8)]:
+                          (4096, 8, 256, 16, 8), (8192, 4, 64, 32, 8),
+                          (200, 8, 64, 8, 8), (256, 2, 8, 8, 64), (1000, 4, 64, 8, 8), (1024, 8, 256, 32, 8)]:
         T -= T % R
         idx = rng.integers(-1, E, size=(T, K)).astype(np.int32)
         ref = oracle.layout(idx, E, R)
