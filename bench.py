@@ -301,7 +301,8 @@ class Workload:
         # batches far larger than L2: one ep_layout_dispatch call with the side stream (C4: 289.5 against 291.2 us
         # per step with separate calls); at C3 the early-resident dispatch CTAs delay the pair half (59.8 against 56.7 us)
         self.one_call_split = self.split_layout and not separate_calls and not is_small(cfg)
-        # decode-size batches: layout and dispatch in one launch (ep_layout_dispatch)
+        # decode-size batches: layout and dispatch in one call (ep_layout_dispatch: the lean layout kernel and a dispatch
+        # launched behind it; the one-launch form only for shapes the lean kernels do not cover)
         self.fused = (not separate_calls) and T <= 1024 and not cfg.host_staged
         self.one_call = one_call and not self.fused and not cfg.host_staged
         if self.one_call:
@@ -322,7 +323,7 @@ class Workload:
             ep.ep_combine(self.out, lay.pair_slot, self.w, self.y, E, R, status=lay.status)
             return
         if self.fused or self.one_call:
-            ep.ep_layout_dispatch(self.idx, self.x, self.recv, E, R, lay, self.ws)    # small batches: one launch for both
+            ep.ep_layout_dispatch(self.idx, self.x, self.recv, E, R, lay, self.ws)    # small batches: one call for both
         elif not self.split_layout:
             ep.ep_layout(self.idx, E, R, out=lay, workspace=self.ws)
         else:
@@ -552,7 +553,7 @@ def measure(ep, wl, steps, warmup, rep, no_graph=False, sample_clocks=True):
         return [e[a].elapsed_time(e[b]) for e in evs]
 
     ops = {"layout": dict(stats_us(span("t0", "t1")),
-                          what="layout and dispatch in one launch (ep_layout_dispatch)" if wl.fused else
+                          what="layout and dispatch in one call (ep_layout_dispatch)" if wl.fused else
                           "whole layout" if not wl.split_layout else "receive-row half (critical path)"),
            "dispatch": dict(stats_us(span("t0", "t2") if wl.fused else span("t1", "t2")), bytes=alg["dispatch"]),
            "combine": dict(stats_us(span("t3", "t4")), bytes=alg["combine"])}
@@ -570,7 +571,7 @@ def measure(ep, wl, steps, warmup, rep, no_graph=False, sample_clocks=True):
                         " inside a graph, each step after a flush"))
     return {"total_ms": total_ms, "step": stats_us(step_ms), "ops": ops, "launches": int(launches), "floor": floor if small else None,
             "n_recv": n_recv, "n_pairs": n_pairs, "alg": alg, "launch": launch_note,
-            "layout": "ep_layout_dispatch (layout and dispatch in one launch)" if wl.fused else
+            "layout": "ep_layout_dispatch (layout kernel and a dependent dispatch launch, one call)" if wl.fused else
             "one ep_layout call" if not wl.split_layout else
             ("ep_layout_dispatch with a second stream (receive-row half, dispatch launched behind it, pair half on the "
              "side stream); the per-kernel pass issues the same work as separate calls" if wl.one_call_split else
@@ -591,7 +592,7 @@ def ops_alone(ep, wl, alg, per_graph=8, replays=4):
     if wl.split_layout:
         calls["layout_receive_row_half"] = lambda: ep.ep_layout_ranks(wl.idx, E, R, lay, wl.ws)
     if wl.fused:
-        calls["layout_dispatch_one_launch"] = lambda: ep.ep_layout_dispatch(wl.idx, wl.x, wl.recv, E, R, lay, wl.ws)
+        calls["layout_dispatch_one_call"] = lambda: ep.ep_layout_dispatch(wl.idx, wl.x, wl.recv, E, R, lay, wl.ws)
     res = {}
     side = torch.cuda.Stream()
     for name, fn in calls.items():

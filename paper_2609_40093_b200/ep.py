@@ -218,8 +218,9 @@ def ep_layout_static_scratch_bytes() -> int:
 
 def ep_layout_dispatch(topk_idx: torch.Tensor, x: torch.Tensor, recv: torch.Tensor, E: int, R: int, out: Layout,
                        workspace: torch.Tensor, stream_pairs=None) -> Layout:
-    """`ep_layout` followed by `ep_dispatch`: one launch for batches of up to 1024 tokens; for larger ones
-    dispatch is launched behind the layout, whose pair half runs on `stream_pairs` (a torch stream) if given."""
+    """`ep_layout` followed by `ep_dispatch` in one call: dispatch is launched behind the layout kernels and loads
+    its rows while they run; past 1024 tokens the layout's pair half runs on `stream_pairs` (a torch stream) if
+    given; small batches of shapes the fastest layout kernels do not cover take a single launch."""
     _want(topk_idx, torch.int32, "topk_idx"), _want(x, torch.bfloat16, "x"), _want(recv, torch.bfloat16, "recv")
     T, K = topk_idx.shape
     st = out.as_struct()

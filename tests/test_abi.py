@@ -114,7 +114,7 @@ def test_host_staged_calls_check_their_segment_tables_before_touching_a_gpu():
     assert per_sender(good, sender_flags=p, timeout=3_000_000_000) == -2      # ... of at most two seconds
     assert L.ep_layout_dispatch(ctypes.byref(ep._shape(T, K, 60, E, R)), p, p, None, p, 16, p, 8, None, None) == -2
     assert L.ep_layout_dispatch(ctypes.byref(shape), None, p, None, p, 16, p, 8, None, None) == -1
-    big = ep._shape(4096, 8, 64, 128, 8)                     # past the one-launch form: a second stream needs two workspaces
+    big = ep._shape(4096, 8, 64, 128, 8)                     # more than 1024 tokens: a second stream needs two workspaces
     one = L.ep_layout_workspace_bytes(ctypes.byref(big))
     lay = ep._Layout(*[256] * 11)
     assert L.ep_layout_dispatch(ctypes.byref(big), p, p, ctypes.byref(lay), p, one, p, 8, None, p) == -3

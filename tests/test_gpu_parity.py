@@ -452,7 +452,7 @@ def test_layout_and_dispatch_in_one_call(T, H, E, K, R, routing):
 
 
 def test_small_step_with_the_fused_call_replays_from_a_cuda_graph():
-    """layout+dispatch in one launch, combine launched with programmatic stream serialisation behind it:
+    """layout+dispatch in one call, combine launched with programmatic stream serialisation behind it:
     captured once, replayed on new inputs."""
     cfg = inputs.CONFIGS["C2"]
     T, K, H, E, R = cfg.T, cfg.K, cfg.H, cfg.E, cfg.R
@@ -635,7 +635,7 @@ def _guarded_layout(T, K, E, R, guard=64, sentinel=-77):
 
 
 def test_layout_writes_nothing_outside_its_output_arrays():
-    """Every form of the layout (one CTA, cluster, two general kernels, lean kernels, the one-launch
+    """Every form of the layout (one CTA, cluster, two general kernels, lean kernels alone and as a pair, the one-launch
     layout + dispatch) with its outputs carved from one guarded buffer: the words between the arrays and
     the entries past N_recv / P keep their sentinel."""
     rng = np.random.default_rng(78)
