@@ -437,16 +437,18 @@ namespace ep {
 namespace {
 
 // ---------------------------------------------------------------- lean form
-// Batches past the one-CTA form with compile-time K and at most RT <= 32 ranks (and, for the pair half, E <= 1024): one token
-// per lane with its picks in registers (vector loads, no staging for the counting), the rank ballots in
-// registers, 256 tokens per CTA. Same two-kernel exchange as the general form, and the same scratch: the first
-// kernel writes cta_part[cta] = [R rank-hit counters | bad ids | E expert counters], the second is launched with programmatic
-// stream serialisation and waits on the device before it reads them -- the rank counters with the whole CTA
-// at once (one L2 round trip, summed by shared-memory atomics: only sums are used), the expert counters one
-// expert per thread. One warp scans the ranks and sets the warps' receive-row bases while another scans the
-// experts; every pick's receive row is looked up by its rank; the slots leave as 16-byte stores. The pair
-// half replays each warp's 32*K pairs in (t,k) order from a staged copy, four 32-pair steps in flight, with
-// warp-private expert counters as in the general form.
+// Compile-time K (1..8 and 10) and at most RT <= 32 ranks (and, for the pair half, E <= 1024): one token per lane
+// with its picks in registers (vector loads, no staging for the counting), the rank ballots in registers, 256
+// tokens per CTA. Up to 256 tokens the main kernel runs alone as one CTA (its own counters are the totals). Beyond,
+// the same two-kernel exchange as the general form: the first kernel writes
+// cta_part[cta] = [R rank-hit counters | bad ids | E expert counters], the second is launched with programmatic
+// stream serialisation and waits on the device before it reads them: it requests its share of the rank counters
+// and then a batch of expert counters (one expert per thread) before it uses either, so that both exchanges share
+// one L2 round trip (the rank counters are summed by shared-memory atomics: only sums are used). In the receive-row
+// half every warp scans the ranks itself and sets its own receive-row bases; in the pair half one warp does that
+// for all while another scans the experts. Every pick's receive row is looked up by its rank; the slots leave as
+// 16-byte stores. The pair half replays each warp's 32*K pairs in (t,k) order from a staged copy, four 32-pair
+// steps in flight, with warp-private expert counters as in the general form.
 //   PAIRS == false: the receive-row half alone (what dispatch waits for), no dynamic shared memory;
 //   PAIRS == true : the pair half, or both halves (a.parts).
 constexpr int kLeanWarps = kLeanTokensPerCta / 32;
@@ -469,17 +471,20 @@ __device__ __forceinline__ void load_picks(const int32_t *idx, int t, int32_t (&
             const int4 v = __ldg(p + i);
             e[4 * i] = v.x; e[4 * i + 1] = v.y; e[4 * i + 2] = v.z; e[4 * i + 3] = v.w;
         }
-    } else {
+    } else if (KT % 2 == 0) {
         const int2 *p = reinterpret_cast<const int2 *>(idx + (size_t)t * KT);
 #pragma unroll
         for (int i = 0; i < KT / 2; ++i) {
             const int2 v = __ldg(p + i);
             e[2 * i] = v.x; e[2 * i + 1] = v.y;
         }
+    } else {
+#pragma unroll
+        for (int i = 0; i < KT; ++i) e[i] = __ldg(idx + (size_t)t * KT + i);
     }
 }
 
-// KT ints of one token to global or shared memory as 16- or 8-byte stores
+// KT ints of one token to global or shared memory as 16- or 8-byte stores (odd KT: one by one)
 template <int KT>
 __device__ __forceinline__ void store_picks(int32_t *dst, const int32_t (&v)[KT])
 {
@@ -487,9 +492,12 @@ __device__ __forceinline__ void store_picks(int32_t *dst, const int32_t (&v)[KT]
 #pragma unroll
         for (int i = 0; i < KT / 4; ++i)
             reinterpret_cast<int4 *>(dst)[i] = make_int4(v[4 * i], v[4 * i + 1], v[4 * i + 2], v[4 * i + 3]);
-    } else {
+    } else if (KT % 2 == 0) {
 #pragma unroll
         for (int i = 0; i < KT / 2; ++i) reinterpret_cast<int2 *>(dst)[i] = make_int2(v[2 * i], v[2 * i + 1]);
+    } else {
+#pragma unroll
+        for (int i = 0; i < KT; ++i) dst[i] = v[i];
     }
 }
 
@@ -806,7 +814,7 @@ int pick_kernels(int K, int R)               // the general kernels: exact (K, R
     return 0;
 }
 
-// The lean kernels: exact K, any rank count up to the bound they were compiled for (8 or 32).
+// The lean kernels: exact K (1..8 and 10), any rank count up to the bound they were compiled for (8 or 32).
 struct LeanKernels {
     LayoutKernel ranks_count, ranks_assign;          // the receive-row half alone
     LayoutKernel count, assign;                      // the pair half, or both halves
@@ -818,20 +826,28 @@ constexpr LeanKernels lean_kernels()
                        lean_assign_kernel<KT, RT, true>};
 }
 constexpr int kLeanRankBounds[] = {8, 32};
-const LeanKernels kLeanKernels[2][4] = {
-    {lean_kernels<2, 8>(), lean_kernels<4, 8>(), lean_kernels<6, 8>(), lean_kernels<8, 8>()},
-    {lean_kernels<2, 32>(), lean_kernels<4, 32>(), lean_kernels<6, 32>(), lean_kernels<8, 32>()}};
+constexpr int kLeanTopK[] = {1, 2, 3, 4, 5, 6, 7, 8, 10};    // 10 of 512: the finest model the paper names
+constexpr int kNumLeanTopK = sizeof(kLeanTopK) / sizeof(int);
+template <int RT>
+struct LeanRow {
+    LeanKernels k[kNumLeanTopK] = {lean_kernels<1, RT>(), lean_kernels<2, RT>(), lean_kernels<3, RT>(), lean_kernels<4, RT>(),
+                                   lean_kernels<5, RT>(), lean_kernels<6, RT>(), lean_kernels<7, RT>(), lean_kernels<8, RT>(),
+                                   lean_kernels<10, RT>()};
+};
+const LeanRow<8> kLeanKernels8;
+const LeanRow<32> kLeanKernels32;
+const LeanKernels *lean_row(int b) { return b == 0 ? kLeanKernels8.k : kLeanKernels32.k; }
 
 const LeanKernels *pick_lean(int K, int R)
 {
     for (int b = 0; b < 2; ++b)
         if (R <= kLeanRankBounds[b])
-            for (int i = 0; i < 4; ++i)
-                if (K == kTunedTopK[i]) return &kLeanKernels[b][i];
+            for (int i = 0; i < kNumLeanTopK; ++i)
+                if (K == kLeanTopK[i]) return &lean_row(b)[i];
     return nullptr;
 }
 
-// Which form a call takes: the lean kernels need an even top-k of at most 8, at most 32 ranks, 16-byte aligned tables
+// Which form a call takes: the lean kernels need a top-k of at most 8 (or 10), at most 32 ranks, 16-byte aligned tables
 // and, for the pair half, at most 1024 experts; the kernel pair also one scratch row per CTA inside the workspace.
 enum { kGeneral = 0, kLeanSingle = 1, kLeanPair = 2 };
 int lean_form(const ep_shape_t &s, const void *topk_idx, const ep_layout_t &out, size_t workspace_bytes, int parts)
@@ -926,9 +942,9 @@ int run_layout(const ep_shape_t *shape, const int32_t *topk_idx, const ep_layout
             EP_CUDA_TRY(cudaFuncSetAttribute(kKernelPairs[i].assign, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget));
         }
         for (int b = 0; b < 2; ++b)
-            for (int i = 0; i < 4; ++i)
-                EP_CUDA_TRY(cudaFuncSetAttribute(kLeanKernels[b][i].assign, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                 (int)lean_smem_bytes(kLeanMaxExperts, kTunedTopK[i])));
+            for (int i = 0; i < kNumLeanTopK; ++i)
+                EP_CUDA_TRY(cudaFuncSetAttribute(lean_row(b)[i].assign, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                 (int)lean_smem_bytes(kLeanMaxExperts, kLeanTopK[i])));
         attr_done[dev].store(true, std::memory_order_release);
     }
     const int which = pick_kernels(shape->top_k, R);

@@ -399,25 +399,29 @@ def test_largest_config_in_full():
     _full_path_check(cfg, d["topk_idx"], d["topk_weights"], d["x"])
 
 
-FUSED = [  # T, H, E, K, R, routing: ep_layout_dispatch on batches that take its one-launch form (odd K, K > 8 or
-           # R > 32, up to 1024 tokens), on batches the lean layout kernels take instead, and on larger ones
-    (64, 256, 8, 2, 2, "uniform"),         # C1
-    (256, 4096, 8, 2, 8, "uniform"),       # C2
+FUSED = [  # T, H, E, K, R, routing: ep_layout_dispatch on batches that take its one-launch form (K = 9 or above 10,
+           # or R > 32, up to 1024 tokens), on batches the lean layout kernels take instead, and on larger ones
+    (64, 256, 8, 2, 2, "uniform"),         # C1: lean main kernel alone + dependent dispatch
+    (256, 4096, 8, 2, 8, "uniform"),       # C2: the same, a full CTA
     (1, 8, 1, 1, 1, "uniform"),
     (2, 16, 2, 1, 2, "uniform"),
     (8, 264, 8, 2, 4, "uniform"),
     (96, 2880, 32, 4, 4, "uniform"),
     (40, 520, 16, 4, 1, "uniform"),        # R = 1, 40 tokens: a ragged last group
     (48, 72, 16, 3, 16, "uniform"),
-    (1000, 136, 512, 10, 8, "zipf"),
+    (1000, 136, 512, 10, 8, "zipf"),       # 10 of 512: four CTAs of the lean kernel pair
     (1024, 7168, 256, 8, 8, "burst"),      # four CTAs of the lean kernel pair, long rows
-    (1024, 7168, 256, 7, 8, "uniform"),    # the largest batch of the one-launch form, long rows
     (520, 72, 64, 6, 8, "zipf"),           # three CTAs of the lean kernel pair, the last one ragged
-    (320, 64, 4096, 4, 64, "uniform"),     # E and R at their maxima
-    (64, 64, 64, 32, 32, "uniform"),       # K at its maximum
     (1023 - 1023 % 3, 40, 24, 5, 3, "zipf_identity"),
-    (1088, 64, 4096, 32, 64, "uniform"),   # does not fit: falls back to the two calls
-    (2048, 24, 128, 6, 8, "zipf"),         # more than 1024 tokens: falls back
+    (1024, 7168, 256, 9, 8, "uniform"),    # one launch: the largest batch of that form, long rows
+    (96, 2880, 36, 9, 4, "uniform"),       # one launch, 360 vectors per row
+    (512, 264, 48, 12, 16, "zipf"),        # one launch, K = 12
+    (40, 520, 16, 11, 1, "uniform"),       # one launch, R = 1, a ragged last group
+    (64, 8, 64, 16, 64, "uniform"),        # one launch, one token per rank
+    (320, 64, 4096, 4, 64, "uniform"),     # one launch, E and R at their maxima
+    (64, 64, 64, 32, 32, "uniform"),       # one launch, K at its maximum
+    (1088, 64, 4096, 32, 64, "uniform"),   # does not fit one launch: falls back to the general kernels
+    (2048, 24, 128, 6, 8, "zipf"),         # more than 1024 tokens
 ]
 
 
@@ -523,14 +527,18 @@ def test_layout_and_dispatch_in_one_call_with_a_second_stream(name):
     assert err.value.code == -3
 
 
-@pytest.mark.parametrize("K", [2, 4, 6, 8])
+LEAN_TOP_K = [1, 2, 3, 4, 5, 6, 7, 8, 10]
+
+
+@pytest.mark.parametrize("K", LEAN_TOP_K)
 def test_receive_row_half_on_the_lean_kernels(K):
-    """ep_layout_ranks with R = 8 and K in {2, 4, 6, 8} past 1024 tokens takes kernels of its own (picks in
-    registers, vector loads and stores). Ragged batch ends, masked / repeated / out-of-range ids, a batch too
-    large for them (falls back), and a routing table that is not 16-byte aligned (falls back)."""
+    """ep_layout_ranks with K in 1..8 or 10 takes kernels of its own (picks in registers, vector loads and
+    stores where K is even): alone as one CTA up to 256 tokens, as a pair beyond. Ragged batch ends, masked /
+    repeated / out-of-range ids, a batch too large for them (falls back), and a routing table that is not
+    16-byte aligned (falls back)."""
     rng = np.random.default_rng(20 + K)
     R, E = 8, 64
-    for T in (1032, 2048, 4096 + 8, 8192, 32768, 40000):
+    for T in (8, 200, 256, 264, 520, 1000, 1032, 2048, 4096 + 8, 8192, 32768, 40000):
         idx = rng.integers(0, E, size=(T, K)).astype(np.int32)
         idx[rng.random((T, K)) < 0.1] = -1
         idx[7, :] = idx[7, 0]
@@ -550,13 +558,13 @@ def test_receive_row_half_on_the_lean_kernels(K):
             assert (lay.pair_slot.cpu().numpy() == -7).all()   # the pair half is not this call's business
 
 
-@pytest.mark.parametrize("K", [2, 4, 6, 8])
+@pytest.mark.parametrize("K", LEAN_TOP_K)
 def test_whole_layout_and_pair_half_on_the_lean_kernels(K):
-    """ep_layout and ep_layout_pairs with R = 8, K in {2, 4, 6, 8} and E <= 1024 past 1024 tokens take the lean
-    kernels too. Ragged batch ends, masked / repeated / out-of-range ids, 1024 experts, a batch and an expert
-    count too large for them (fall back), and a routing table that is not 16-byte aligned (falls back)."""
+    """ep_layout and ep_layout_pairs with K in 1..8 or 10 and E <= 1024 take the lean kernels too. Ragged batch
+    ends, masked / repeated / out-of-range ids, 1024 experts, a batch and an expert count too large for them
+    (fall back), and a routing table that is not 16-byte aligned (falls back)."""
     rng = np.random.default_rng(40 + K)
-    for T, E, R in ((1032, 64, 8), (2048, 8, 8), (4096 + 8, 128, 8), (8192, 256, 8), (32768, 1024, 8), (40000, 64, 8),
+    for T, E, R in ((8, 8, 8), (96, 1024, 32), (256, 64, 8), (264, 64, 8), (520, 256, 8), (1000, 40, 5), (1032, 64, 8), (2048, 8, 8), (4096 + 8, 128, 8), (8192, 256, 8), (32768, 1024, 8), (40000, 64, 8),
                     (2048, 2048, 8), (3000, 30, 1), (3000, 30, 2), (4098, 63, 3), (2052, 12, 4), (2051 * 5 // 5 * 5, 35, 5),
                     (4200, 49, 7), (2048, 48, 16), (4096 + 32, 1024, 32), (6144, 96, 24), (2048, 128, 64)):
         T -= T % R
