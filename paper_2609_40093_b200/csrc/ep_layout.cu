@@ -13,8 +13,9 @@
 //   4. replays its tiles in (t,k) order with running counters that start at
 //      offset[bin] + earlier CTAs + earlier warps of this CTA.
 // Step 2 has three forms:
-//   single   one CTA of up to 32 warps holds every tile (up to 1024 tokens): nothing
-//            to exchange, one launch;
+//   single   one CTA of up to 8 warps holds every tile (up to 256 tokens): nothing
+//            to exchange, one launch (32 warps on one SM took 26 us for 1024 tokens,
+//            four CTAs of 8 warps take 12);
 //   cluster  up to 8 CTAs of 8 warps (up to 2048 tokens) form one thread-block cluster
 //            and read each other's CTA totals through distributed shared memory
 //            between two cluster barriers: one launch, no global scratch;
@@ -47,7 +48,7 @@ namespace cg = cooperative_groups;
 namespace ep {
 namespace {
 
-constexpr int kMaxWarpsSingle = 32;     // one CTA holds every tile: up to 1024 tokens
+constexpr int kMaxWarpsSingle = 8;      // one CTA holds every tile: up to 256 tokens
 constexpr int kMaxWarps = 8;            // warps per CTA otherwise (the replay's scattered stores are bound per SM: spread it)
 constexpr int kMaxCluster = 8;          // portable cluster size
 constexpr int kMaxCtasGlobal = 128;
