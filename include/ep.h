@@ -138,11 +138,10 @@ int ep_layout_pairs(const ep_shape_t *shape, const int32_t *topk_idx, const ep_l
  * provides topk_idx and every output array.
  *
  *   - Limit: the scratch a shape needs is ep_layout_workspace_bytes(shape): 16
- *     bytes while the batch fits one thread-block cluster (2048 tokens, fewer
- *     when large E or K shrink the CTA), else 4*(E+R+1) bytes per CTA, at most
- *     128 CTAs (34 KB for T=8192, E=256, R=8). Shapes
- *     that need more than the array holds return EP_ERR_STATIC_SCRATCH and
- *     enqueue nothing.
+ *     bytes up to 256 tokens, else 4*(E+R+1) bytes per CTA of 256 tokens (fewer
+ *     tokens when large E or K shrink the CTA, more once there would be over
+ *     128 CTAs; 34 KB for T=8192, E=256, R=8). Shapes that need more than the
+ *     array holds return EP_ERR_STATIC_SCRATCH and enqueue nothing.
  *   - First call on a device: looks up the array's device address (once per
  *     device, with that device current). Make that first call outside any
  *     stream capture.
