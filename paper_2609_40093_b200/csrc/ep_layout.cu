@@ -53,7 +53,7 @@ constexpr int kMaxWarps = 8;            // warps per CTA otherwise (the replay's
 constexpr int kMaxCluster = 8;          // portable cluster size
 constexpr int kMaxCtasGlobal = 128;
 constexpr size_t kSmemBudget = 200 * 1024;
-constexpr int kSteps = 4;               // 32-pair steps of the replay whose latencies overlap
+constexpr int kSteps = 2;               // 32-pair steps of the replay whose latencies overlap (4 in flight: 1 us slower at T=8192)
 
 enum { kModeSingle = 0, kModeCluster = 1, kModeGlobal = 2 };
 enum { kPartRanks = 1, kPartPairs = 2 };
@@ -448,12 +448,12 @@ namespace {
 // one L2 round trip (the rank counters are summed by shared-memory atomics: only sums are used). In the receive-row
 // half every warp scans the ranks itself and sets its own receive-row bases; in the pair half one warp does that
 // for all while another scans the experts. Every pick's receive row is looked up by its rank; the slots leave as
-// 16-byte stores. The pair half replays each warp's 32*K pairs in (t,k) order from a staged copy, four 32-pair
+// 16-byte stores. The pair half replays each warp's 32*K pairs in (t,k) order from a staged copy, two 32-pair
 // steps in flight, with warp-private expert counters as in the general form.
 //   PAIRS == false: the receive-row half alone (what dispatch waits for), no dynamic shared memory;
 //   PAIRS == true : the pair half, or both halves (a.parts).
 constexpr int kLeanWarps = kLeanTokensPerCta / 32;
-constexpr int kLeanSteps = 4;
+constexpr int kLeanSteps = 2;                     // 32-pair steps of the replay in flight (8.3 us per call at C4; 8.9 with 1, 9.6 with 4, 10.4 with 8)
 constexpr int kLeanExchangeBatch = 32;              // CTAs' expert counters a thread requests at once
 
 inline size_t lean_smem_bytes(int E, int K)
