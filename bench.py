@@ -668,6 +668,31 @@ def time_variants(ep, wl, n_recv, n_pairs, iters=20):
     return res
 
 
+def duplex_link_probe(dev, nbytes=256 << 20, reps=5):
+    """One host-to-device and one device-to-host cudaMemcpyAsync of `nbytes` each (pinned), on two streams at the
+    same time: GB/s per direction, best of `reps`. What the host link gives when both directions are busy."""
+    h_up, h_dn = torch.empty(nbytes, dtype=torch.uint8).pin_memory(), torch.empty(nbytes, dtype=torch.uint8).pin_memory()
+    d_up, d_dn = torch.empty(nbytes, dtype=torch.uint8, device=dev), torch.zeros(nbytes, dtype=torch.uint8, device=dev)
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    best = 1e30
+    for _ in range(reps + 1):
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e1, e2 = torch.cuda.Event(), torch.cuda.Event()
+        a.record()
+        s1.wait_event(a), s2.wait_event(a)
+        with torch.cuda.stream(s1):
+            d_up.copy_(h_up, non_blocking=True)
+        with torch.cuda.stream(s2):
+            h_dn.copy_(d_dn, non_blocking=True)
+        e1.record(s1), e2.record(s2)
+        torch.cuda.current_stream().wait_event(e1), torch.cuda.current_stream().wait_event(e2)
+        b.record()
+        torch.cuda.synchronize()
+        best = min(best, a.elapsed_time(b))
+    return nbytes / (best * 1e-3) / 1e9
+
+
 def host_staged_arms(ep, wl, iters=10, sweep=True):
     """Receive buffer in mapped pinned host memory: (i) the dispatch kernel stores straight
     into it; (ii) dispatch packs into device staging and the copy engine moves each rank's
@@ -707,7 +732,8 @@ def host_staged_arms(ep, wl, iters=10, sweep=True):
     def arm_copy_blind():           # no count reaches the host: one copy of the worst-case T*min(K,R) rows
         ep.ep_dispatch_copy_engine(x, lay.recv_slot, staging, recv_host, E, R, rank_row_offsets_host=None)
 
-    res = {"host_link_d2h_GB/s": d2h, "host_link_h2d_GB/s": h2d, "rows": n_recv, "bytes_over_link": n_recv * row}
+    res = {"host_link_d2h_GB/s": d2h, "host_link_h2d_GB/s": h2d,
+           "host_link_duplex_GB/s_each_way": duplex_link_probe(dev), "rows": n_recv, "bytes_over_link": n_recv * row}
     for name, fn, nbytes in [("kernel_store", arm_kernel, n_recv * row),
                              ("copy_engine_per_rank", arm_copy_known, n_recv * row),
                              ("copy_engine_worst_case", arm_copy_blind, recv_host.shape[0] * row)]:
@@ -911,12 +937,17 @@ def main():
     y_h = torch.empty(T, H, dtype=torch.bfloat16).pin_memory()
     st_h = torch.zeros(1, dtype=torch.int32).pin_memory()
     n_e2e = max(1, args.e2e_steps)
-    e2e_chunks = 8 if T >= 2048 else 1
+    e2e_chunks = 2 if T >= 2048 else 1       # C4, steps back to back: 2.61 ms with 2 chunks, 2.64 with 4, 2.78 with 8
     s_in, s_comp, s_out = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()
 
+    step_events, e2e_round = ep.StepEvents(), [0]
+
     def e2e_step():
+        # consecutive steps alternate between two copies of the arena's transfer buffers: a step's uploads run
+        # while the previous step's results are still on their way back
         ep.ep_host_step_pipelined(wl.x_h, wl.idx_h, wl.w_h, y_h, arena, E, R, e2e_chunks, s_in, s_comp, s_out,
-                                  status_host=st_h)
+                                  status_host=st_h, round=e2e_round[0], step_events=step_events)
+        e2e_round[0] += 1
 
     torch.cuda.synchronize()
     for _ in range(3 if args.e2e_steps > 0 else 0):
@@ -935,6 +966,7 @@ def main():
     h2d = wl.x_h.numel() * 2 + wl.idx_h.numel() * 4 + wl.w_h.numel() * 4
     d2h = y_h.numel() * 2 + 4
     del arena
+    duplex = duplex_link_probe(dev) if args.e2e_steps > 0 else None    # both directions busy: the ceiling of the e2e step
 
     # the library's own stream probes on this GPU, beside the measured copy peak
     probes = None
@@ -989,7 +1021,11 @@ def main():
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": e2e_ms / n_e2e, "steps": args.e2e_steps,
                 "call": f"ep_host_step_pipelined (layout+dispatch+group+combine, pinned host in/out, {e2e_chunks} token "
-                        "chunk(s) on upload/compute/download streams)"},
+                        "chunk(s) on upload/compute/download streams; consecutive steps alternate between two copies "
+                        "of the arena's transfer buffers, so a step's uploads overlap the previous step's downloads)",
+                "link_GB/s_each_way": (h2d / (e2e_ms / n_e2e * 1e-3) / 1e9) if args.e2e_steps > 0 else None,
+                "link_duplex_probe_GB/s_each_way": duplex if args.e2e_steps > 0 else None,
+                "frac_of_duplex_probe": (h2d / (e2e_ms / n_e2e * 1e-3) / 1e9 / duplex) if args.e2e_steps > 0 else None},
         "gpu_launches": m["launches"],
         "context": CONTEXT,
     }

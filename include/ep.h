@@ -425,11 +425,24 @@ int ep_host_step(const ep_shape_t *shape, const void *x_host, const int32_t *top
  * (the call orders itself after the previous one). 1 <= chunks <= 256. Ordering
  * events come from the library's process-wide pool (see the host-staged
  * conventions above); calls from several host threads are serialised.
+ * Steps back to back (Section 4.4: two buffers used in turn, so that a round's
+ * transfers need not wait for the round before it): the arena holds two copies
+ * of what the copy streams touch (x, topk_idx, topk_weights, y, the status
+ * word). With step_events == NULL every call uses the first copy and waits for
+ * the previous call's kernels before it uploads and for its downloads before it
+ * computes. With step_events = four caller-owned cudaEvent_t (created by the
+ * caller, never recorded or recorded long ago; the same four for every call on
+ * this arena) call number `round` (0, 1, 2, ... consecutive) uses copy
+ * round & 1 and waits only for call round - 2, which used the same copy:
+ * its uploads start while the previous call's downloads are still running. The
+ * call records step_events[round & 1] behind its kernels and
+ * step_events[2 + (round & 1)] behind its downloads. Errors: EP_ERR_NULL for a
+ * NULL entry of step_events, EP_ERR_INVALID_ARG for round < 0.
  */
 int ep_host_step_pipelined(const ep_shape_t *shape, const void *x_host, const int32_t *topk_idx_host,
                            const float *topk_weights_host, void *y_host, int32_t *status_host, void *arena,
                            size_t arena_bytes, int chunks, void *stream_in, void *stream_compute,
-                           void *stream_out);
+                           void *stream_out, int round, void *const *step_events);
 
 /* Reads a device status word: copies it to *status_host and SYNCHRONISES the stream. */
 int ep_status(const int32_t *status_dev, void *stream, int32_t *status_host);

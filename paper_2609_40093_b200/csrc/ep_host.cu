@@ -110,7 +110,10 @@ struct StepBuffers {
     size_t total;
 };
 
-StepBuffers carve_step(const ep_shape_t &s, void *arena)
+// `half` picks one of the two copies of what the copy streams touch (x, topk_idx, topk_weights, y and the
+// status word), so that a step's uploads and downloads need not wait for the step before it; everything else
+// is used on the compute stream only and is ordered by it.
+StepBuffers carve_step(const ep_shape_t &s, void *arena, int half = 0)
 {
     StepBuffers b;
     const size_t T = s.num_tokens, K = s.top_k, H = s.hidden, E = s.num_experts, R = s.num_ranks;
@@ -118,12 +121,17 @@ StepBuffers carve_step(const ep_shape_t &s, void *arena)
     Carver c(arena);
     b.recv_rows = (int64_t)rows;
     b.pair_rows = (int64_t)TK;
-    b.x = c.take<uint16_t>(T * H);
+    for (int h = 0; h < 2; ++h) {
+        uint16_t *x = c.take<uint16_t>(T * H), *y = c.take<uint16_t>(T * H);
+        int32_t *idx = c.take<int32_t>(TK);
+        float *w = c.take<float>(TK);
+        int32_t *status = c.take<int32_t>(1);
+        if (h == half) {
+            b.x = x; b.y = y; b.idx = idx; b.w = w; b.lay.status = status;
+        }
+    }
     b.recv = c.take<uint16_t>(rows * H);
     b.grouped = c.take<uint16_t>(TK * H);
-    b.y = c.take<uint16_t>(T * H);
-    b.idx = c.take<int32_t>(TK);
-    b.w = c.take<float>(TK);
     b.lay.expert_counts = c.take<int32_t>(E);
     b.lay.expert_offsets = c.take<int32_t>(E + 1);
     b.lay.rank_rows = c.take<int32_t>(R);
@@ -134,7 +142,6 @@ StepBuffers carve_step(const ep_shape_t &s, void *arena)
     b.lay.recv_token = c.take<int32_t>(rows);
     b.lay.pair_row = c.take<int32_t>(TK);
     b.lay.pair_token = c.take<int32_t>(TK);
-    b.lay.status = c.take<int32_t>(1);
     b.workspace_bytes = ep_layout_workspace_bytes(&s);
     b.workspace = c.take<char>(b.workspace_bytes);
     b.total = c.used;
@@ -222,14 +229,16 @@ extern "C" int ep_host_step(const ep_shape_t *shape, const void *x_host, const i
 extern "C" int ep_host_step_pipelined(const ep_shape_t *shape, const void *x_host, const int32_t *topk_idx_host,
                                       const float *topk_weights_host, void *y_host, int32_t *status_host,
                                       void *arena, size_t arena_bytes, int chunks, void *stream_in_,
-                                      void *stream_compute_, void *stream_out_)
+                                      void *stream_compute_, void *stream_out_, int round, void *const *step_events)
 {
     using namespace ep;
     int rc = check_shape(shape, true);
     if (rc != EP_OK) return rc;
     if (!arena) return EP_ERR_NULL;
-    if ((reinterpret_cast<uintptr_t>(arena) & 255u) != 0 || chunks < 1 || chunks > 256) return EP_ERR_INVALID_ARG;
-    const StepBuffers b = carve_step(*shape, arena);
+    if ((reinterpret_cast<uintptr_t>(arena) & 255u) != 0 || chunks < 1 || chunks > 256 || round < 0) return EP_ERR_INVALID_ARG;
+    if (step_events && (!step_events[0] || !step_events[1] || !step_events[2] || !step_events[3])) return EP_ERR_NULL;
+    const int half = step_events ? (round & 1) : 0;
+    const StepBuffers b = carve_step(*shape, arena, half);
     if (arena_bytes < b.total) return EP_ERR_CAPACITY;
     if (shape->num_tokens == 0) return EP_OK;
     if (!x_host || !topk_idx_host || !topk_weights_host || !y_host) return EP_ERR_NULL;
@@ -240,12 +249,19 @@ extern "C" int ep_host_step_pipelined(const ep_shape_t *shape, const void *x_hos
     rc = order_events(&ev, 2 * chunks + 3, hold);
     if (rc != EP_OK) return rc;
     const size_t T = shape->num_tokens, K = shape->top_k, H = shape->hidden;
-    // the arena is reused from step to step: uploads wait for the previous step's kernels, and the
-    // kernels for the previous step's downloads of y
-    EP_CUDA_TRY(cudaEventRecord(ev[0], comp));
-    EP_CUDA_TRY(cudaStreamWaitEvent(in, ev[0], 0));
-    EP_CUDA_TRY(cudaEventRecord(ev[1], outs));
-    EP_CUDA_TRY(cudaStreamWaitEvent(comp, ev[1], 0));
+    if (step_events) {
+        // this half of the arena was last used two steps ago: its uploads wait for that step's kernels and its
+        // kernels for that step's downloads, not for the step before this one, whose transfers are still running
+        EP_CUDA_TRY(cudaStreamWaitEvent(in, static_cast<cudaEvent_t>(step_events[half]), 0));
+        EP_CUDA_TRY(cudaStreamWaitEvent(comp, static_cast<cudaEvent_t>(step_events[2 + half]), 0));
+    } else {
+        // one half, reused from step to step: uploads wait for the previous step's kernels, and the kernels
+        // for the previous step's downloads of y
+        EP_CUDA_TRY(cudaEventRecord(ev[0], comp));
+        EP_CUDA_TRY(cudaStreamWaitEvent(in, ev[0], 0));
+        EP_CUDA_TRY(cudaEventRecord(ev[1], outs));
+        EP_CUDA_TRY(cudaStreamWaitEvent(comp, ev[1], 0));
+    }
     EP_CUDA_TRY(cudaMemcpyAsync(b.idx, topk_idx_host, T * K * sizeof(int32_t), cudaMemcpyHostToDevice, in));
     EP_CUDA_TRY(cudaMemcpyAsync(b.w, topk_weights_host, T * K * sizeof(float), cudaMemcpyHostToDevice, in));
     EP_CUDA_TRY(cudaEventRecord(ev[2], in));
@@ -278,6 +294,10 @@ extern "C" int ep_host_step_pipelined(const ep_shape_t *shape, const void *x_hos
     }
     if (status_host)
         EP_CUDA_TRY(cudaMemcpyAsync(status_host, b.lay.status, sizeof(int32_t), cudaMemcpyDeviceToHost, outs));
+    if (step_events) {
+        EP_CUDA_TRY(cudaEventRecord(static_cast<cudaEvent_t>(step_events[half]), comp));
+        EP_CUDA_TRY(cudaEventRecord(static_cast<cudaEvent_t>(step_events[2 + half]), outs));
+    }
     return EP_OK;
 }
 

@@ -89,7 +89,7 @@ def lib() -> ctypes.CDLL:
         L.ep_host_step_arena_bytes.restype = sz
         L.ep_host_step_arena_bytes.argtypes = [sp]
         L.ep_host_step.argtypes = [sp, vp, vp, vp, vp, vp, vp, sz, vp]
-        L.ep_host_step_pipelined.argtypes = [sp, vp, vp, vp, vp, vp, vp, sz, i32, vp, vp, vp]
+        L.ep_host_step_pipelined.argtypes = [sp, vp, vp, vp, vp, vp, vp, sz, i32, vp, vp, vp, i32, vp]
         L.ep_host_step_pipelined.restype = i32
         L.ep_status.argtypes = [vp, vp, vp]
         L.ep_probe_bandwidth.argtypes = [i32, vp, vp, sz, i32, vp, ctypes.POINTER(ctypes.c_double)]
@@ -385,16 +385,32 @@ def ep_host_step(x_host, topk_idx_host, topk_weights_host, y_host, arena, E, R, 
     return y_host
 
 
+class StepEvents:
+    """Four caller-owned CUDA events for `ep_host_step_pipelined` calls back to back on one arena (kernels done and
+    downloads done, per copy of the arena's transfer buffers). torch creates an event's handle when it is first
+    recorded, so all four are recorded once on the current stream here."""
+
+    def __init__(self):
+        self.events = [torch.cuda.Event() for _ in range(4)]
+        for e in self.events:
+            e.record()
+        self.array = (ctypes.c_void_p * 4)(*[ctypes.c_void_p(e.cuda_event) for e in self.events])
+
+
 def ep_host_step_pipelined(x_host, topk_idx_host, topk_weights_host, y_host, arena, E, R, chunks, stream_in,
-                           stream_compute, stream_out, status_host=None):
-    """`ep_host_step` with uploads, kernels and downloads of token chunks overlapping on three streams."""
+                           stream_compute, stream_out, status_host=None, round=0, step_events: StepEvents = None):
+    """`ep_host_step` with uploads, kernels and downloads of token chunks overlapping on three streams. With
+    `step_events` consecutive calls (round = 0, 1, 2, ...) alternate between two copies of the arena's transfer
+    buffers, so that a call's uploads overlap the previous call's downloads."""
     T, H = x_host.shape
     K = topk_idx_host.shape[1]
     _check(lib().ep_host_step_pipelined(ctypes.byref(_shape(T, K, H, E, R)), _ptr(x_host), _ptr(topk_idx_host),
                                         _ptr(topk_weights_host), _ptr(y_host), _ptr(status_host), _ptr(arena),
                                         arena.numel(), int(chunks), ctypes.c_void_p(stream_in.cuda_stream),
                                         ctypes.c_void_p(stream_compute.cuda_stream),
-                                        ctypes.c_void_p(stream_out.cuda_stream)), "ep_host_step_pipelined")
+                                        ctypes.c_void_p(stream_out.cuda_stream), int(round),
+                                        None if step_events is None else ctypes.cast(step_events.array, ctypes.c_void_p)),
+           "ep_host_step_pipelined")
     return y_host
 
 

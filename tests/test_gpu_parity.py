@@ -368,6 +368,39 @@ def test_pipelined_host_step_matches_oracle(chunks):
         np.testing.assert_array_equal(yh.view(torch.int16).numpy().view(np.uint16), want)
 
 
+@pytest.mark.parametrize("chunks", [1, 4])
+def test_pipelined_host_steps_alternate_between_two_copies_of_the_transfer_buffers(chunks):
+    """Five different batches back to back with caller-owned step events and no synchronisation: call n uses
+    copy n & 1 of x / topk_idx / topk_weights / y / status and waits only for call n - 2. Every result and
+    every status word (one batch carries an id outside [-1, E)) against the oracle."""
+    cfg = inputs.CONFIGS["C3"]
+    hosts, wants = [], []
+    for seed in range(5):
+        d = inputs.make_inputs(cfg, seed)
+        idx, w, x = d["topk_idx"].copy(), d["topk_weights"], d["x"]
+        if seed == 2:
+            idx[17, 3] = cfg.E + 5
+        ref = oracle.layout(idx, cfg.E, cfg.R)
+        recv = oracle.dispatch(x, ref.recv_slot, ref.n_recv)
+        wants.append((oracle.combine_f32(recv[ref.pair_row], ref.pair_slot, w), ref.status))
+        hosts.append((torch.from_numpy(x.view(np.int16)).view(torch.bfloat16).pin_memory(),
+                      torch.from_numpy(idx).pin_memory(), torch.from_numpy(w).pin_memory(),
+                      torch.zeros(cfg.T, cfg.H, dtype=torch.bfloat16).pin_memory(),
+                      torch.full((1,), -1, dtype=torch.int32).pin_memory()))
+    arena = torch.empty(ep.ep_host_step_arena_bytes(cfg.T, cfg.K, cfg.H, cfg.E, cfg.R), dtype=torch.uint8, device="cuda")
+    s_in, s_comp, s_out = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()
+    events = ep.StepEvents()
+    torch.cuda.synchronize()
+    for n, (xh, ih, wh, yh, sh) in enumerate(hosts):
+        ep.ep_host_step_pipelined(xh, ih, wh, yh, arena, cfg.E, cfg.R, chunks, s_in, s_comp, s_out, status_host=sh,
+                                  round=n, step_events=events)
+    torch.cuda.synchronize()
+    for (xh, ih, wh, yh, sh), (want, status) in zip(hosts, wants):
+        assert int(sh[0]) == status
+        np.testing.assert_array_equal(yh.view(torch.int16).numpy().view(np.uint16), want)
+    assert wants[2][1] == ep.STATUS_BAD_INDEX
+
+
 def test_host_staged_dispatch_both_arms():
     """Receive buffer in mapped pinned host memory: kernel stores and the copy-engine arm."""
     cfg = inputs.CONFIGS["C5"]
