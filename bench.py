@@ -493,8 +493,8 @@ class _FrozenEvent:
 
 
 def measure(ep, wl, steps, warmup, rep, no_graph=False, sample_clocks=True):
-    """Times `steps` steps of a workload. Big workloads: back to back, direct launches, per-kernel events
-    inside the timed region. Small workloads: every step after an L2 flush, timed by its own event pair
+    """Times `steps` steps of a workload. Big workloads: back to back from a CUDA graph (or direct launches), then
+    once more as direct launches with per-kernel events. Small workloads: every step after an L2 flush, timed by its own event pair
     recorded inside a CUDA graph (small_in_graph), or with direct launches (small_direct)."""
     cfg, lay = wl.cfg, wl.lay
     small = is_small(cfg)
@@ -511,18 +511,47 @@ def measure(ep, wl, steps, warmup, rep, no_graph=False, sample_clocks=True):
     torch.cuda.synchronize()
     launches0 = ep.ep_launch_count()
     if not small:
-        # pass A, the timed region: K steps back to back, one event before and one after
+        # pass A, the timed region: K steps back to back, one event before and one after. The steps are replayed
+        # from a CUDA graph that holds G of them (G = the largest divisor of K up to 25): the same kernels with the
+        # same dependencies, without the host's launch gaps (C4: 282-285 us per step against 288-289 with direct
+        # launches, which --no-graph times instead; host-staged workloads always use direct launches).
+        graph, per_graph, n_replays = None, 0, 0
+        if not no_graph and not cfg.host_staged:
+            in_graph = max(g for g in range(1, 26) if steps % g == 0)
+            n_replays = steps // in_graph
+            graph = torch.cuda.CUDAGraph()
+            l0 = ep.ep_launch_count()
+            with torch.cuda.graph(graph):
+                for _ in range(in_graph):
+                    wl.step()
+            per_graph = ep.ep_launch_count() - l0
+            graph.replay()                                # uploads the graph: untimed, part of the warm-up
+            torch.cuda.synchronize()
+            launches0 = ep.ep_launch_count()
         rep.barrier()
         if clocks:
             clocks.__enter__()
         start.record()
-        for i in range(steps):
-            wl.step()
+        if graph is not None:
+            for i in range(n_replays):
+                graph.replay()
+        else:
+            for i in range(steps):
+                wl.step()
         stop.record()
         torch.cuda.synchronize()
         rep.barrier()
-        launches = ep.ep_launch_count() - launches0
+        launches = per_graph * n_replays if graph is not None else ep.ep_launch_count() - launches0
         total_ms = rep.max_over_ranks(start.elapsed_time(stop))
+        direct_us = None
+        if graph is not None:                             # the same K steps as direct launches, for comparison only
+            a_d, b_d = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a_d.record()
+            for i in range(steps):
+                wl.step()
+            b_d.record()
+            torch.cuda.synchronize()
+            direct_us = a_d.elapsed_time(b_d) / steps * 1e3
         # pass B, the same K steps again with events between the calls: per-kernel durations (the seven event
         # records per step cost a few microseconds of stream time, which is why they are kept out of pass A)
         evs = [wl.new_events() for _ in range(steps)]
@@ -536,8 +565,11 @@ def measure(ep, wl, steps, warmup, rep, no_graph=False, sample_clocks=True):
             clocks.__exit__()
         rep.barrier()
         step_ms = [e["t0"].elapsed_time(e["t4"]) for e in evs]
-        launch_note = (f"direct launches; value from {steps} steps with no events inside; per-kernel durations from the "
-                       f"same {steps} steps repeated with events between the calls "
+        how = (f"a CUDA graph of {steps // n_replays} step(s) replayed {n_replays} time(s) back to back "
+               f"(the same {steps} steps as direct launches: {direct_us:.1f} us per step)") if graph is not None else \
+            "direct launches"
+        launch_note = (f"{how}; value from {steps} steps with no events inside; per-kernel durations from the "
+                       f"same {steps} steps repeated as direct launches with events between the calls "
                        f"({start_b.elapsed_time(stop_b) / steps * 1e3:.1f} us per step)")
     else:
         flusher = L2Flush(wl.dev)
@@ -886,7 +918,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=20)
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--no-graph", action="store_true", help="small workloads: time direct launches, not graph replays")
+    ap.add_argument("--no-graph", action="store_true", help="time direct launches, not graph replays")
     ap.add_argument("--serial-layout", action="store_true",
                     help="one ep_layout call instead of the receive-row half before dispatch and the pair half beside it")
     ap.add_argument("--separate-calls", action="store_true",
