@@ -243,6 +243,51 @@ def test_whole_step_replays_from_a_cuda_graph():
         assert ep.ep_status(lay.status) == 0
 
 
+def test_two_stream_steps_replay_from_one_cuda_graph():
+    """The form the benchmark times: three steps back to back, each one `ep_layout_dispatch` with a second
+    stream (pair half of the layout beside dispatch, joined by the library's events) and a combine launched
+    behind it, captured in one CUDA graph and replayed on new inputs. The last step's outputs against the oracle."""
+    cfg = inputs.CONFIGS["C3"]
+    T, K, H, E, R = cfg.T, cfg.K, cfg.H, cfg.E, cfg.R
+    idx_d = torch.zeros(T, K, dtype=torch.int32, device="cuda")
+    w_d = torch.zeros(T, K, dtype=torch.float32, device="cuda")
+    x_d = torch.zeros(T, H, dtype=torch.bfloat16, device="cuda")
+    out_d = torch.zeros(T * K, H, dtype=torch.bfloat16, device="cuda")
+    lay = ep.alloc_layout(T, K, E, R)
+    ws = torch.empty(2 * ep.ep_layout_workspace_bytes(T, K, E, R) + 256, dtype=torch.uint8, device="cuda")
+    recv = torch.zeros(T * min(K, R), H, dtype=torch.bfloat16, device="cuda")
+    y = torch.zeros(T, H, dtype=torch.bfloat16, device="cuda")
+    pairs_stream = torch.cuda.Stream()
+
+    def step():
+        ep.ep_layout_dispatch(idx_d, x_d, recv, E, R, lay, ws, stream_pairs=pairs_stream)
+        ep.ep_combine(out_d, lay.pair_slot, w_d, y, E, R, status=lay.status)
+
+    warm = torch.cuda.Stream()
+    with torch.cuda.stream(warm):
+        step()
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        for _ in range(3):
+            step()
+    for seed in (5, 6):
+        d = inputs.make_inputs(cfg, seed)
+        out = inputs.make_out(cfg, T * K, seed=seed)
+        idx_d.copy_(torch.from_numpy(d["topk_idx"]))
+        w_d.copy_(torch.from_numpy(d["topk_weights"]))
+        x_d.copy_(dev_bf16(d["x"]))
+        out_d.copy_(dev_bf16(out))
+        recv.zero_(), y.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        ref = oracle.layout(d["topk_idx"], E, R)
+        assert_layout_equal(lay, ref)
+        np.testing.assert_array_equal(host_bits(recv)[:ref.n_recv], oracle.dispatch(d["x"], ref.recv_slot, ref.n_recv))
+        np.testing.assert_array_equal(host_bits(y), oracle.combine_f32(out, ref.pair_slot, d["topk_weights"]))
+        assert ep.ep_status(lay.status) == 0
+
+
 def test_empty_batch():
     E, R, K, H = 8, 2, 2, 64
     lay = ep.alloc_layout(0, K, E, R, fill=-7)
