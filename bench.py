@@ -874,6 +874,25 @@ def host_staged_arms(ep, wl, iters=10, sweep=True):
         rounds[name] = {"us_per_round": best * 1e3 / n_rounds, "rounds": n_rounds,
                         "GB/s_each_way": 2 * n_recv * row * n_rounds / (best * 1e-3) / 1e9}
     res["dispatch_plus_combine_rounds"] = rounds
+    # independent dispatch round trips back to back: what the two alternating bounce halves are for
+    n_trips = 8
+    trips_b2b = {}
+    for name, overlap in [("ordered by the download stream", False), ("overlapped (per-half events)", True)]:
+        best = 1e30
+        for _ in range(3):
+            hf = ep.HalfFreeEvents() if overlap else None
+            torch.cuda.synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(up)
+            for rnd in range(n_trips):
+                ep.ep_host_roundtrip(x, lay.recv_slot, offs_host, staging, bounce, back, E, R, round=rnd, chunks_per_rank=1,
+                                     duplex=True, stream_up=up, stream_down=down, half_free=hf)
+            b.record(down)
+            torch.cuda.synchronize()
+            best = min(best, a.elapsed_time(b))
+        trips_b2b[name] = {"us_per_trip": best * 1e3 / n_trips, "trips": n_trips,
+                           "GB/s_each_way": n_recv * row * n_trips / (best * 1e-3) / 1e9}
+    res["dispatch_roundtrips_back_to_back"] = trips_b2b
     return res
 
 
