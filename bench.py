@@ -553,14 +553,36 @@ def measure(ep, wl, steps, warmup, rep, no_graph=False, sample_clocks=True):
             torch.cuda.synchronize()
             direct_us = a_d.elapsed_time(b_d) / steps * 1e3
         # pass B, the same K steps again with events between the calls: per-kernel durations (the seven event
-        # records per step cost a few microseconds of stream time, which is why they are kept out of pass A)
-        evs = [wl.new_events() for _ in range(steps)]
+        # records per step cost a few microseconds of stream time, which is why they are kept out of pass A).
+        # Replayed from a graph like pass A (events recorded inside it), or direct launches.
         start_b, stop_b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        start_b.record()
-        for i in range(steps):
-            wl.step(evs[i])
-        stop_b.record()
-        torch.cuda.synchronize()
+        if graph is not None:
+            ops_evs = [wl.new_events(external=True) for _ in range(steps // n_replays)]
+            g_ops = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g_ops):
+                for e in ops_evs:
+                    wl.step(e)
+            g_ops.replay()
+            torch.cuda.synchronize()
+            spans = [("t0", "t1"), ("t1", "t2"), ("t0", "t2"), ("t2", "t3"), ("t3", "t4"), ("t0", "t4")]
+            if wl.split_layout:
+                spans.append(("p0", "p1"))
+            evs, pass_b_ms = [], 0.0
+            for _ in range(n_replays):
+                start_b.record()
+                g_ops.replay()
+                stop_b.record()
+                torch.cuda.synchronize()
+                pass_b_ms += start_b.elapsed_time(stop_b)
+                evs += [FrozenEvents({(a, b): e[a].elapsed_time(e[b]) for a, b in spans}) for e in ops_evs]
+        else:
+            evs = [wl.new_events() for _ in range(steps)]
+            start_b.record()
+            for i in range(steps):
+                wl.step(evs[i])
+            stop_b.record()
+            torch.cuda.synchronize()
+            pass_b_ms = start_b.elapsed_time(stop_b)
         if clocks:
             clocks.__exit__()
         rep.barrier()
@@ -569,8 +591,8 @@ def measure(ep, wl, steps, warmup, rep, no_graph=False, sample_clocks=True):
                f"(the same {steps} steps as direct launches: {direct_us:.1f} us per step)") if graph is not None else \
             "direct launches"
         launch_note = (f"{how}; value from {steps} steps with no events inside; per-kernel durations from the "
-                       f"same {steps} steps repeated as direct launches with events between the calls "
-                       f"({start_b.elapsed_time(stop_b) / steps * 1e3:.1f} us per step)")
+                       f"same {steps} steps repeated in the same way with events between the calls "
+                       f"({pass_b_ms / steps * 1e3:.1f} us per step)")
     else:
         flusher = L2Flush(wl.dev)
         floor = None
