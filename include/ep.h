@@ -179,8 +179,8 @@ int ep_dispatch(const ep_shape_t *shape, const void *x, const int32_t *recv_slot
  * kernel, launched so that its CTAs load their rows of x while the layout still
  * runs (x and topk_idx are inputs of this call: they must be complete on
  * `stream` before it). Only batches of up to 1024 tokens that the layout's
- * fastest kernels do not cover (a top-k of 9 or above 10, more than 32
- * ranks, tables that are not 16-byte aligned) and whose routing table fits in
+ * fastest kernels do not cover (a top-k of 9 or above 10, more than 1024
+ * experts, tables that are not 16-byte aligned) and whose routing table fits in
  * shared memory take one launch in which every CTA derives the layout for itself
  * and moves its own tokens' rows. stream_pairs (may be NULL) is a second
  * stream for batches of more than 1024 tokens: the pair half of the layout,

@@ -438,7 +438,8 @@ namespace ep {
 namespace {
 
 // ---------------------------------------------------------------- lean form
-// Compile-time K (1..8 and 10) and at most RT <= 32 ranks (and, for the pair half, E <= 1024): one token per lane
+// Compile-time K (1..8 and 10), a compile-time bound RT on the ranks (8, 32 or 64; 64 is the library's limit) and, for
+// the pair half, E <= 1024: one token per lane
 // with its picks in registers (vector loads, no staging for the counting), the rank ballots in registers, 256
 // tokens per CTA. Up to 256 tokens the main kernel runs alone as one CTA (its own counters are the totals). Beyond,
 // the same two-kernel exchange as the general form: the first kernel writes
@@ -502,17 +503,27 @@ __device__ __forceinline__ void store_picks(int32_t *dst, const int32_t (&v)[KT]
     }
 }
 
+// rank bitmask of a token: 32 bits up to 32 ranks, 64 beyond
+template <int RT>
+struct RankMask {
+    using type = unsigned;
+};
+template <>
+struct RankMask<64> {
+    using type = unsigned long long;
+};
+
 // picks -> ranks (or -1), rank bitmask, number of ids outside [-1, E)
-template <int KT>
-__device__ __forceinline__ unsigned picks_to_ranks(const LayoutArgs &a, const int32_t (&e)[KT], int (&rk)[KT], int *bad)
+template <int KT, typename Mask>
+__device__ __forceinline__ Mask picks_to_ranks(const LayoutArgs &a, const int32_t (&e)[KT], int (&rk)[KT], int *bad)
 {
-    unsigned mask = 0u;
+    Mask mask = 0;
 #pragma unroll
     for (int k = 0; k < KT; ++k) {
         rk[k] = -1;
         if ((unsigned)e[k] < (unsigned)a.E) {
             rk[k] = sdiv(e[k], a.mul_El);
-            mask |= 1u << rk[k];
+            mask |= Mask(1) << rk[k];
         } else if (e[k] != -1) {
             ++*bad;
         }
@@ -536,20 +547,24 @@ __global__ void __launch_bounds__(kLeanWarps * 32) lean_count_kernel(LayoutArgs 
 #pragma unroll
     for (int k = 0; k < KT; ++k) e[k] = -1;
     if (t < a.T) load_picks<KT>(a.idx, t, e);
-    const unsigned mask = picks_to_ranks<KT>(a, e, rk, &bad);
+    using Mask = typename RankMask<RT>::type;
+    constexpr int kRanksPerLane = (RT + 31) / 32;    // lane l counts ranks l, l + 32
+    const Mask mask = picks_to_ranks<KT, Mask>(a, e, rk, &bad);
     __syncthreads();
     if (PAIRS) {
 #pragma unroll
         for (int k = 0; k < KT; ++k)
             if (rk[k] >= 0) atomicAdd(dyn + e[k], 1);
     }
-    int mine = 0;
+    int mine[kRanksPerLane] = {};
 #pragma unroll
     for (int r = 0; r < RT; ++r) {
-        const int c = __popc(__ballot_sync(kFullMask, (mask >> r) & 1u));
-        if (lane == r) mine = c;
+        const int c = __popc(__ballot_sync(kFullMask, (unsigned)(mask >> r) & 1u));
+        if (lane == (r & 31)) mine[r >> 5] = c;
     }
-    if (lane < RT && mine) atomicAdd(cnt + lane, mine);
+#pragma unroll
+    for (int j = 0; j < kRanksPerLane; ++j)
+        if (lane + 32 * j < RT && mine[j]) atomicAdd(cnt + lane + 32 * j, mine[j]);
     if (bad) atomicAdd(cnt + RT, bad);
     __syncthreads();
     // one row per CTA, as wide as the general form's: [R rank-hit counters | bad ids | E expert counters]
@@ -590,14 +605,18 @@ __global__ void __launch_bounds__(kLeanWarps * 32) lean_assign_kernel(LayoutArgs
 #pragma unroll
     for (int k = 0; k < KT; ++k) e[k] = -1;
     if (t < a.T) load_picks<KT>(a.idx, t, e);
-    const unsigned mask = picks_to_ranks<KT>(a, e, rk, &bad);
-    unsigned bal[RT];
+    using Mask = typename RankMask<RT>::type;
+    constexpr int kRanksPerLane = (RT + 31) / 32;    // lane l scans ranks l, l + 32
+    constexpr bool kKeepBallots = RT <= 32;          // the ballots stay in registers too, or only in shared memory
+    const Mask mask = picks_to_ranks<KT, Mask>(a, e, rk, &bad);
+    unsigned bal[kKeepBallots ? RT : 1];
 #pragma unroll
     for (int r = 0; r < RT; ++r) {
-        bal[r] = __ballot_sync(kFullMask, (mask >> r) & 1u);
-        if (lane == r) {
-            wcnt[warp][r] = __popc(bal[r]);
-            bal_s[warp][r] = bal[r];
+        const unsigned b = __ballot_sync(kFullMask, (unsigned)(mask >> r) & 1u);
+        if (kKeepBallots) bal[kKeepBallots ? r : 0] = b;
+        if (lane == (r & 31)) {
+            wcnt[warp][r] = __popc(b);
+            bal_s[warp][r] = b;
         }
     }
     if (PAIRS) {
@@ -677,39 +696,55 @@ __global__ void __launch_bounds__(kLeanWarps * 32) lean_assign_kernel(LayoutArgs
     // PAIRS: warp 1 scans the ranks and sets every warp's bases while warp 0 scans the experts. Otherwise every warp
     // scans the ranks itself and sets its own bases: no serial section, no second block barrier.
     if (!PAIRS || warp == 1) {
-        // lane r < R: rank r (RT <= 32 ranks fit one warp); acc[.][RT] holds the ids outside [-1, E)
-        const int32_t before = lane < R ? acc[0][lane] : 0, hits = lane < R ? acc[1][lane] : 0;
-        int32_t incl = hits;                         // scan over ranks: rank_row_offsets
+        // lane l: ranks l and (RT = 64) l + 32; acc[.][RT] holds the ids outside [-1, E)
+        int32_t before[kRanksPerLane], hits[kRanksPerLane], incl[kRanksPerLane];
+        int32_t carry = 0;                           // hits of the ranks below this lane's j-th rank's block of 32
 #pragma unroll
-        for (int off = 1; off < 32; off <<= 1) {
-            const int32_t up = __shfl_up_sync(kFullMask, incl, off);
-            if (lane >= off) incl += up;
+        for (int j = 0; j < kRanksPerLane; ++j) {
+            const int r = lane + 32 * j;
+            before[j] = r < R ? acc[0][r] : 0;
+            hits[j] = r < R ? acc[1][r] : 0;
+            int32_t x = hits[j];                     // scan over ranks: rank_row_offsets
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const int32_t up = __shfl_up_sync(kFullMask, x, off);
+                if (lane >= off) x += up;
+            }
+            incl[j] = x + carry;
+            carry = __shfl_sync(kFullMask, incl[j], 31);
         }
-        const int32_t offset = incl - hits;
-        const int32_t n_recv = __shfl_sync(kFullMask, incl, 31);
+        const int32_t n_recv = carry;
         if (blockIdx.x == 0 && ranks && (PAIRS || warp == 0)) {
-            if (lane < R) {
-                a.out.rank_rows[lane] = hits;
-                a.out.rank_row_offsets[lane] = offset;
-                a.out.src_row_offsets[lane * (R + 1) + R] = incl;
+#pragma unroll
+            for (int j = 0; j < kRanksPerLane; ++j) {
+                const int r = lane + 32 * j;
+                if (r < R) {
+                    a.out.rank_rows[r] = hits[j];
+                    a.out.rank_row_offsets[r] = incl[j] - hits[j];
+                    a.out.src_row_offsets[r * (R + 1) + R] = incl[j];
+                }
             }
             if (lane == 0) {
                 a.out.rank_row_offsets[R] = n_recv;
                 *a.out.status = acc[1][RT] ? EP_STATUS_BAD_INDEX : 0;
             }
         }
-        if (lane < RT) {
-            int32_t run = offset + before;
-            if (PAIRS) {
 #pragma unroll
-                for (int w = 0; w < kLeanWarps; ++w) {
-                    base[w][lane] = run;
-                    run += wcnt[w][lane];
+        for (int j = 0; j < kRanksPerLane; ++j) {
+            const int r = lane + 32 * j;
+            if (r < RT) {
+                int32_t run = incl[j] - hits[j] + before[j];
+                if (PAIRS) {
+#pragma unroll
+                    for (int w = 0; w < kLeanWarps; ++w) {
+                        base[w][r] = run;
+                        run += wcnt[w][r];
+                    }
+                } else {
+#pragma unroll
+                    for (int w = 0; w < kLeanWarps - 1; ++w) run += w < warp ? wcnt[w][r] : 0;
+                    base[warp][r] = run;
                 }
-            } else {
-#pragma unroll
-                for (int w = 0; w < kLeanWarps - 1; ++w) run += w < warp ? wcnt[w][lane] : 0;
-                base[warp][lane] = run;
             }
         }
     }
@@ -740,8 +775,8 @@ __global__ void __launch_bounds__(kLeanWarps * 32) lean_assign_kernel(LayoutArgs
         const bool first_of_source = t == s * a.Tr;  // where source rank s's segment starts in every rank
 #pragma unroll
         for (int r = 0; r < RT; ++r) {
-            const int32_t row = base[warp][r] + __popc(bal[r] & lt);
-            if ((mask >> r) & 1u) a.out.recv_token[row] = t;   // a rank's rows of these 32 tokens are consecutive
+            const int32_t row = base[warp][r] + __popc((kKeepBallots ? bal[kKeepBallots ? r : 0] : bal_s[warp][r]) & lt);
+            if ((unsigned)(mask >> r) & 1u) a.out.recv_token[row] = t;   // a rank's rows of these 32 tokens are consecutive
             if (first_of_source && r < R) a.out.src_row_offsets[r * (R + 1) + s] = row;
         }
     }
@@ -815,7 +850,7 @@ int pick_kernels(int K, int R)               // the general kernels: exact (K, R
     return 0;
 }
 
-// The lean kernels: exact K (1..8 and 10), any rank count up to the bound they were compiled for (8 or 32).
+// The lean kernels: exact K (1..8 and 10), any rank count up to the bound they were compiled for (8, 32 or 64).
 struct LeanKernels {
     LayoutKernel ranks_count, ranks_assign;          // the receive-row half alone
     LayoutKernel count, assign;                      // the pair half, or both halves
@@ -826,7 +861,8 @@ constexpr LeanKernels lean_kernels()
     return LeanKernels{lean_count_kernel<KT, RT, false>, lean_assign_kernel<KT, RT, false>, lean_count_kernel<KT, RT, true>,
                        lean_assign_kernel<KT, RT, true>};
 }
-constexpr int kLeanRankBounds[] = {8, 32};
+constexpr int kLeanRankBounds[] = {8, 32, 64};
+constexpr int kNumLeanRankBounds = 3;
 constexpr int kLeanTopK[] = {1, 2, 3, 4, 5, 6, 7, 8, 10};    // 10 of 512: the finest model the paper names
 constexpr int kNumLeanTopK = sizeof(kLeanTopK) / sizeof(int);
 template <int RT>
@@ -837,18 +873,19 @@ struct LeanRow {
 };
 const LeanRow<8> kLeanKernels8;
 const LeanRow<32> kLeanKernels32;
-const LeanKernels *lean_row(int b) { return b == 0 ? kLeanKernels8.k : kLeanKernels32.k; }
+const LeanRow<64> kLeanKernels64;
+const LeanKernels *lean_row(int b) { return b == 0 ? kLeanKernels8.k : b == 1 ? kLeanKernels32.k : kLeanKernels64.k; }
 
 const LeanKernels *pick_lean(int K, int R)
 {
-    for (int b = 0; b < 2; ++b)
+    for (int b = 0; b < kNumLeanRankBounds; ++b)
         if (R <= kLeanRankBounds[b])
             for (int i = 0; i < kNumLeanTopK; ++i)
                 if (K == kLeanTopK[i]) return &lean_row(b)[i];
     return nullptr;
 }
 
-// Which form a call takes: the lean kernels need a top-k of at most 8 (or 10), at most 32 ranks, 16-byte aligned tables
+// Which form a call takes: the lean kernels need a top-k of at most 8 (or 10), 16-byte aligned tables
 // and, for the pair half, at most 1024 experts; the kernel pair also one scratch row per CTA inside the workspace.
 enum { kGeneral = 0, kLeanSingle = 1, kLeanPair = 2 };
 int lean_form(const ep_shape_t &s, const void *topk_idx, const ep_layout_t &out, size_t workspace_bytes, int parts)
@@ -942,7 +979,7 @@ int run_layout(const ep_shape_t *shape, const int32_t *topk_idx, const ep_layout
             EP_CUDA_TRY(cudaFuncSetAttribute(kKernelPairs[i].count, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget));
             EP_CUDA_TRY(cudaFuncSetAttribute(kKernelPairs[i].assign, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBudget));
         }
-        for (int b = 0; b < 2; ++b)
+        for (int b = 0; b < kNumLeanRankBounds; ++b)
             for (int i = 0; i < kNumLeanTopK; ++i)
                 EP_CUDA_TRY(cudaFuncSetAttribute(lean_row(b)[i].assign, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                  (int)lean_smem_bytes(kLeanMaxExperts, kLeanTopK[i])));

@@ -615,8 +615,9 @@ def test_receive_row_half_on_the_lean_kernels(K):
     repeated / out-of-range ids, a batch too large for them (falls back), and a routing table that is not
     16-byte aligned (falls back)."""
     rng = np.random.default_rng(20 + K)
-    R, E = 8, 64
-    for T in (8, 200, 256, 264, 520, 1000, 1032, 2048, 4096 + 8, 8192, 32768, 40000):
+    cases = [(T, 8, 64) for T in (8, 200, 256, 264, 520, 1000, 1032, 2048, 4096 + 8, 8192, 32768, 40000)]
+    cases += [(64, 64, 64), (192, 64, 128), (1024, 64, 256), (8192, 64, 256), (2000, 40, 80), (4096, 32, 64), (33 * 70, 33, 66)]
+    for T, R, E in cases:
         idx = rng.integers(0, E, size=(T, K)).astype(np.int32)
         idx[rng.random((T, K)) < 0.1] = -1
         idx[7, :] = idx[7, 0]
@@ -642,7 +643,8 @@ def test_whole_layout_and_pair_half_on_the_lean_kernels(K):
     ends, masked / repeated / out-of-range ids, 1024 experts, a batch and an expert count too large for them
     (fall back), and a routing table that is not 16-byte aligned (falls back)."""
     rng = np.random.default_rng(40 + K)
-    for T, E, R in ((8, 8, 8), (96, 1024, 32), (256, 64, 8), (264, 64, 8), (520, 256, 8), (1000, 40, 5), (1032, 64, 8), (2048, 8, 8), (4096 + 8, 128, 8), (8192, 256, 8), (32768, 1024, 8), (40000, 64, 8),
+    for T, E, R in ((8, 8, 8), (96, 1024, 32), (256, 64, 8), (264, 64, 8), (520, 256, 8), (1000, 40, 5), (1032, 64, 8),
+                    (64, 64, 64), (192, 128, 64), (512, 256, 64), (8192, 256, 64), (4096 + 64, 1024, 64), (4800, 96, 48), (33 * 70, 66, 33), (2048, 8, 8), (4096 + 8, 128, 8), (8192, 256, 8), (32768, 1024, 8), (40000, 64, 8),
                     (2048, 2048, 8), (3000, 30, 1), (3000, 30, 2), (4098, 63, 3), (2052, 12, 4), (2051 * 5 // 5 * 5, 35, 5),
                     (4200, 49, 7), (2048, 48, 16), (4096 + 32, 1024, 32), (6144, 96, 24), (2048, 128, 64)):
         T -= T % R
@@ -678,7 +680,8 @@ def test_layout_stays_inside_its_workspace():
     for T, K, E, R in [(512, 2, 8, 8), (2048, 6, 128, 8), (1536, 3, 12, 4), (3000, 2, 30, 1), (4098, 2, 63, 3), (8192, 8, 256, 8),
                        (4096, 4, 1024, 8), (4096, 8, 2048, 8), (40000, 2, 16, 8), (3200, 32, 4096, 64), (4200, 6, 49, 7),
                        (4096, 8, 256, 16), (8192, 4, 64, 32), (3000, 6, 60, 20),
-                       (200, 8, 256, 8), (256, 2, 8, 8), (264, 6, 1024, 8), (1000, 4, 64, 8), (1024, 8, 256, 32)]:
+                       (200, 8, 256, 8), (256, 2, 8, 8), (264, 6, 1024, 8), (1000, 4, 64, 8), (1024, 8, 256, 32),
+                       (4096, 8, 256, 64), (320, 4, 128, 64), (2400, 5, 96, 48)]:
         T -= T % R
         idx = rng.integers(-1, E, size=(T, K)).astype(np.int32)
         ref = oracle.layout(idx, E, R)
@@ -728,7 +731,8 @@ def test_layout_writes_nothing_outside_its_output_arrays():
     for T, K, E, R, H in [(96, 3, 12, 4, 64), (1000, 10, 512, 8, 64), (2048, 5, 40, 8, 8), (4096, 8, 128, 8, 8),
                           (3000, 2, 30, 1, 8), (4098, 6, 63, 3, 8), (9000, 7, 64, 4, 8), (40000, 2, 16, 8, 8),
                           (4096, 8, 256, 16, 8), (8192, 4, 64, 32, 8),
-                          (200, 8, 64, 8, 8), (256, 2, 8, 8, 64), (1000, 4, 64, 8, 8), (1024, 8, 256, 32, 8)]:
+                          (200, 8, 64, 8, 8), (256, 2, 8, 8, 64), (1000, 4, 64, 8, 8), (1024, 8, 256, 32, 8),
+                          (4096, 8, 256, 64, 8), (320, 4, 128, 64, 8), (2400, 5, 96, 48, 8)]:
         T -= T % R
         idx = rng.integers(-1, E, size=(T, K)).astype(np.int32)
         ref = oracle.layout(idx, E, R)
