@@ -438,7 +438,7 @@ namespace ep {
 namespace {
 
 // ---------------------------------------------------------------- lean form
-// Compile-time K (1..8 and 10), a compile-time bound RT on the ranks (8, 32 or 64; 64 is the library's limit) and, for
+// Compile-time K (1..8 and 10), a compile-time bound RT on the ranks (8, 16, 32 or 64; 64 is the library's limit) and, for
 // the pair half, E <= 1024: one token per lane
 // with its picks in registers (vector loads, no staging for the counting), the rank ballots in registers, 256
 // tokens per CTA. Up to 256 tokens the main kernel runs alone as one CTA (its own counters are the totals). Beyond,
@@ -650,13 +650,14 @@ __global__ void __launch_bounds__(kLeanWarps * 32) lean_assign_kernel(LayoutArgs
         }
     } else {
         pdl_wait();                                      // cta_part is complete and visible
-        // rank counters of every CTA: the first two per thread are requested here and summed (shared-memory atomics) behind
-        // the expert counters' batch, so that both exchanges share one L2 round trip
+        // rank counters of every CTA: the first kRankBatch per thread are requested here and summed (shared-memory
+        // atomics) behind the expert counters' batch, so that both exchanges share one L2 round trip
+        constexpr int kRankBatch = RT <= 8 ? 2 : RT <= 16 ? 3 : RT <= 32 ? 5 : 9;    // 32 CTAs x (RT + 1) counters over 256 threads
         const int n_items = a.n_ctas * (R + 1);
-        int32_t rv[2];
-        int rc[2], rr[2];
+        int32_t rv[kRankBatch];
+        int rc[kRankBatch], rr[kRankBatch];
 #pragma unroll
-        for (int u = 0; u < 2; ++u) {
+        for (int u = 0; u < kRankBatch; ++u) {
             const int i = min(tid + u * kLeanWarps * 32, n_items - 1);
             rc[u] = sdiv(i, a.mul_R1);
             rr[u] = i - rc[u] * (R + 1);
@@ -675,14 +676,14 @@ __global__ void __launch_bounds__(kLeanWarps * 32) lean_assign_kernel(LayoutArgs
             }
         }
 #pragma unroll
-        for (int u = 0; u < 2; ++u) {
+        for (int u = 0; u < kRankBatch; ++u) {
             const int slot = rr[u] < R ? rr[u] : RT;     // the counter behind the ranks holds the bad ids
             if (tid + u * kLeanWarps * 32 < n_items && rv[u]) {
                 atomicAdd(&acc[1][slot], rv[u]);
                 if (rc[u] < (int)blockIdx.x) atomicAdd(&acc[0][slot], rv[u]);
             }
         }
-        for (int i = tid + 2 * kLeanWarps * 32; i < n_items; i += kLeanWarps * 32) {    // more than 512 counters: the rest
+        for (int i = tid + kRankBatch * kLeanWarps * 32; i < n_items; i += kLeanWarps * 32) {    // more counters: the rest
             const int c = sdiv(i, a.mul_R1), r = i - c * (R + 1);
             const int32_t v = __ldcg(a.cta_part + (size_t)c * stride + r);
             const int slot = r < R ? r : RT;
@@ -850,7 +851,7 @@ int pick_kernels(int K, int R)               // the general kernels: exact (K, R
     return 0;
 }
 
-// The lean kernels: exact K (1..8 and 10), any rank count up to the bound they were compiled for (8, 32 or 64).
+// The lean kernels: exact K (1..8 and 10), any rank count up to the bound they were compiled for (8, 16, 32 or 64).
 struct LeanKernels {
     LayoutKernel ranks_count, ranks_assign;          // the receive-row half alone
     LayoutKernel count, assign;                      // the pair half, or both halves
@@ -861,8 +862,8 @@ constexpr LeanKernels lean_kernels()
     return LeanKernels{lean_count_kernel<KT, RT, false>, lean_assign_kernel<KT, RT, false>, lean_count_kernel<KT, RT, true>,
                        lean_assign_kernel<KT, RT, true>};
 }
-constexpr int kLeanRankBounds[] = {8, 32, 64};
-constexpr int kNumLeanRankBounds = 3;
+constexpr int kLeanRankBounds[] = {8, 16, 32, 64};
+constexpr int kNumLeanRankBounds = 4;
 constexpr int kLeanTopK[] = {1, 2, 3, 4, 5, 6, 7, 8, 10};    // 10 of 512: the finest model the paper names
 constexpr int kNumLeanTopK = sizeof(kLeanTopK) / sizeof(int);
 template <int RT>
@@ -872,9 +873,13 @@ struct LeanRow {
                                    lean_kernels<10, RT>()};
 };
 const LeanRow<8> kLeanKernels8;
+const LeanRow<16> kLeanKernels16;
 const LeanRow<32> kLeanKernels32;
 const LeanRow<64> kLeanKernels64;
-const LeanKernels *lean_row(int b) { return b == 0 ? kLeanKernels8.k : b == 1 ? kLeanKernels32.k : kLeanKernels64.k; }
+const LeanKernels *lean_row(int b)
+{
+    return b == 0 ? kLeanKernels8.k : b == 1 ? kLeanKernels16.k : b == 2 ? kLeanKernels32.k : kLeanKernels64.k;
+}
 
 const LeanKernels *pick_lean(int K, int R)
 {
