@@ -108,7 +108,7 @@ def algorithmic_bytes(cfg, n_recv, n_pairs):
 class ClockSampler:
     """Samples SM clock and throttle reasons of one GPU through NVML while a region runs."""
 
-    def __init__(self, device_index: int, period_s: float = 0.02):
+    def __init__(self, device_index: int, period_s: float = 0.002):
         self.samples, self.reasons = [], set()
         self.max_mhz = None
         self._stop = threading.Event()
